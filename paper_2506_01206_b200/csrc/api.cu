@@ -1,0 +1,278 @@
+// C ABI of the library: argument checks, launch planning, dispatch.  No allocation, no global state.
+#include <limits.h>
+
+#include "commit.cuh"
+#include "common.cuh"
+#include "prefill.cuh"
+#include "tree_step.cuh"
+
+using namespace mdraft;
+
+namespace {
+
+constexpr int kSmCount = 148;  // B200
+
+inline size_t elem_size(int act) { return act == MDRAFT_BF16 ? 2 : 4; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int check_layer(const mdraft_layer* L) {
+    if (!L || !L->A || !L->conv_w) return MDRAFT_ERR_INVALID_ARG;
+    if (L->d_inner <= 0) return MDRAFT_ERR_INVALID_ARG;
+    if (L->d_state != kN || L->d_conv != kW || (L->d_inner % 8) != 0) return MDRAFT_ERR_UNSUPPORTED;
+    if (L->act != MDRAFT_F32 && L->act != MDRAFT_BF16) return MDRAFT_ERR_UNSUPPORTED;
+    if ((L->flags & MDRAFT_PRECONV) && (L->flags & MDRAFT_CONV_ONLY)) return MDRAFT_ERR_INVALID_ARG;
+    if (!aligned16(L->A) || !aligned16(L->conv_w)) return MDRAFT_ERR_MISALIGNED;
+    return MDRAFT_OK;
+}
+
+int check_cache(const mdraft_cache* c, int d_inner, int act, int layer_index) {
+    if (!c || !c->ssm || !c->conv) return MDRAFT_ERR_INVALID_ARG;
+    if (c->n_layers <= 0 || c->n_slots <= 0 || layer_index < 0 || layer_index >= c->n_layers) return MDRAFT_ERR_INVALID_ARG;
+    const int64_t ssm_elems = (int64_t)d_inner * kN, conv_elems = (int64_t)(kW - 1) * d_inner;
+    if (c->ssm_slot_stride < ssm_elems || c->conv_slot_stride < conv_elems) return MDRAFT_ERR_INVALID_ARG;
+    if (c->n_layers > 1 && (c->ssm_layer_stride < 0 || c->conv_layer_stride < 0)) return MDRAFT_ERR_INVALID_ARG;
+    const size_t es = elem_size(act);
+    if (!aligned16(c->ssm) || !aligned16(c->conv)) return MDRAFT_ERR_MISALIGNED;
+    if ((c->ssm_slot_stride * 4) % 16 || (c->ssm_layer_stride * 4) % 16 || (c->conv_slot_stride * es) % 16 ||
+        (c->conv_layer_stride * es) % 16)
+        return MDRAFT_ERR_MISALIGNED;
+    return MDRAFT_OK;
+}
+
+int check_matrix(const void* p, int64_t ld, int cols, int act, bool required) {
+    if (!p) return required ? MDRAFT_ERR_INVALID_ARG : MDRAFT_OK;
+    if (ld < cols) return MDRAFT_ERR_INVALID_ARG;
+    if (!aligned16(p) || (ld * (int64_t)elem_size(act)) % 16) return MDRAFT_ERR_MISALIGNED;
+    return MDRAFT_OK;
+}
+
+LayerDev layer_dev(const mdraft_layer* L) {
+    LayerDev d;
+    d.A = L->A; d.D = L->D; d.conv_w = L->conv_w; d.conv_b = L->conv_b; d.dt_bias = L->dt_bias;
+    d.d_inner = L->d_inner; d.flags = L->flags;
+    return d;
+}
+
+PoolDev pool_dev(const mdraft_cache* c, int act, int layer_index) {
+    PoolDev p;
+    p.ssm = c->ssm + (int64_t)layer_index * c->ssm_layer_stride;
+    p.conv = static_cast<char*>(c->conv) + (int64_t)layer_index * c->conv_layer_stride * (int64_t)elem_size(act);
+    p.ssm_slot_stride = c->ssm_slot_stride;
+    p.conv_slot_stride = c->conv_slot_stride;
+    p.n_slots = c->n_slots;
+    return p;
+}
+
+struct PrefillPlan {
+    int chunk_len;       // tokens per chunk (INT_MAX/2 when every sequence is one chunk)
+    int n_chunks_bound;  // upper bound on the number of chunks
+    bool chunked;
+    size_t off_h, off_sd, off_conv, bytes;
+};
+
+// Chunk length: split the token axis only as far as needed to give every SM a few blocks.
+PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen, const mdraft_prefill_opts* opts) {
+    PrefillPlan pl;
+    int Lc;
+    if (opts && opts->chunk_len > 0) {
+        Lc = opts->chunk_len < 4 ? 4 : opts->chunk_len;
+    } else {
+        const int ch_blocks = (L->d_inner + kPrefillThreads - 1) / kPrefillThreads;
+        const int want = (kSmCount * 4 + ch_blocks - 1) / ch_blocks;
+        Lc = (T + want - 1) / want;
+        if (Lc < 64) Lc = 64;
+        Lc = (Lc + 31) / 32 * 32;
+    }
+    pl.chunked = Lc < max_seqlen;
+    if (!pl.chunked) {
+        pl.chunk_len = INT_MAX / 2;
+        pl.n_chunks_bound = n_seq;
+        pl.off_h = pl.off_sd = pl.off_conv = 0;
+        pl.bytes = 0;
+        return pl;
+    }
+    pl.chunk_len = Lc;
+    pl.n_chunks_bound = n_seq + T / Lc;
+    const size_t D = (size_t)L->d_inner;
+    pl.off_h = 0;
+    pl.off_sd = align_up(pl.off_h + (size_t)pl.n_chunks_bound * D * kN * sizeof(float), 256);
+    pl.off_conv = align_up(pl.off_sd + (size_t)pl.n_chunks_bound * D * sizeof(float), 256);
+    pl.bytes = align_up(pl.off_conv + (size_t)n_seq * (kW - 1) * D * elem_size(L->act), 256);
+    return pl;
+}
+
+__global__ void classify_A_kernel(const float* A, int D, int N, int32_t* res) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= D * N) return;
+    int d = i / N, n = i % N;
+    float a0 = A[(size_t)d * N], a = A[i];
+    if (a != (float)(n + 1) * a0) atomicOr(res + 0, 1);
+    if (!(a <= 0.0f)) atomicOr(res + 1, 1);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* mdraft_status_string(int status) {
+    switch (status) {
+        case MDRAFT_OK: return "ok";
+        case MDRAFT_ERR_INVALID_ARG: return "invalid argument";
+        case MDRAFT_ERR_UNSUPPORTED: return "unsupported shape or dtype (need d_state=16, d_conv=4, d_inner%8==0, fp32/bf16)";
+        case MDRAFT_ERR_MISALIGNED: return "pointer or stride not a multiple of 16 bytes";
+        case MDRAFT_ERR_WORKSPACE: return "workspace missing or too small";
+        case MDRAFT_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+int mdraft_version(void) { return 100; }
+
+size_t mdraft_prefill_workspace_bytes(const mdraft_layer* layer, int32_t total_tokens, int32_t n_seq, int32_t max_seqlen,
+                                      const mdraft_prefill_opts* opts) {
+    if (check_layer(layer) != MDRAFT_OK || total_tokens <= 0 || n_seq <= 0 || max_seqlen <= 0) return 0;
+    return plan_prefill(layer, total_tokens, n_seq, max_seqlen, opts).bytes;
+}
+
+int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cache, int32_t layer_index,
+                             const void* x, int64_t ldx, const void* z, int64_t ldz, const void* dt, int64_t lddt,
+                             const void* B, int64_t ldb, const void* C, int64_t ldc, void* out, int64_t ldo,
+                             int32_t total_tokens, int32_t n_seq, int32_t max_seqlen, const int32_t* cu_seqlens,
+                             const int32_t* init_slot, const int32_t* final_slot, void* workspace, size_t workspace_bytes,
+                             const mdraft_prefill_opts* opts, int32_t* dev_status, void* stream) {
+    int rc = check_layer(layer);
+    if (rc) return rc;
+    if (total_tokens < 0 || n_seq < 0 || max_seqlen < 0) return MDRAFT_ERR_INVALID_ARG;
+    if (opts) {
+        if (opts->chunk_len < 0) return MDRAFT_ERR_INVALID_ARG;
+        for (int i = 0; i < 7; ++i)
+            if (opts->reserved[i]) return MDRAFT_ERR_INVALID_ARG;
+    }
+    const bool needs_pool = init_slot || final_slot;
+    if (needs_pool || cache) {
+        rc = check_cache(cache, layer->d_inner, layer->act, layer_index);
+        if (rc) return rc;
+    }
+    if (n_seq == 0 || total_tokens == 0) {
+        if (n_seq > 0 && !cu_seqlens) return MDRAFT_ERR_INVALID_ARG;
+        if (n_seq == 0) return MDRAFT_OK;
+    }
+    if (!cu_seqlens) return MDRAFT_ERR_INVALID_ARG;
+    const bool conv_only = layer->flags & MDRAFT_CONV_ONLY;
+    const int D = layer->d_inner, act = layer->act;
+    const bool have_rows = total_tokens > 0;
+    if ((rc = check_matrix(x, ldx, D, act, have_rows))) return rc;
+    if ((rc = check_matrix(out, ldo, D, act, have_rows))) return rc;
+    if ((rc = check_matrix(z, ldz, D, act, have_rows && !conv_only))) return rc;
+    if ((rc = check_matrix(dt, lddt, D, act, have_rows && !conv_only))) return rc;
+    if ((rc = check_matrix(B, ldb, kN, act, have_rows && !conv_only))) return rc;
+    if ((rc = check_matrix(C, ldc, kN, act, have_rows && !conv_only))) return rc;
+    if (max_seqlen < 1) max_seqlen = 1;
+
+    PrefillPlan pl = plan_prefill(layer, total_tokens > 0 ? total_tokens : 1, n_seq, max_seqlen, opts);
+    if (pl.chunked) {
+        if (!workspace || workspace_bytes < pl.bytes) return MDRAFT_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MDRAFT_ERR_MISALIGNED;
+    }
+    PrefillArgs a;
+    a.L = layer_dev(layer);
+    if (cache) a.pool = pool_dev(cache, act, layer_index);
+    else { a.pool.ssm = nullptr; a.pool.conv = nullptr; a.pool.ssm_slot_stride = 0; a.pool.conv_slot_stride = 0; a.pool.n_slots = 0; }
+    a.x = x; a.z = z; a.dt = dt; a.B = B; a.C = C; a.out = out;
+    a.ldx = ldx; a.ldz = ldz; a.lddt = lddt; a.ldb = ldb; a.ldc = ldc; a.ldo = ldo;
+    a.T = total_tokens; a.n_seq = n_seq; a.chunk_len = pl.chunk_len; a.n_chunks_bound = pl.n_chunks_bound;
+    a.cu = cu_seqlens; a.init_slot = init_slot; a.final_slot = final_slot;
+    char* ws = static_cast<char*>(workspace);
+    a.ws_h = pl.chunked ? reinterpret_cast<float*>(ws + pl.off_h) : nullptr;
+    a.ws_sd = pl.chunked ? reinterpret_cast<float*>(ws + pl.off_sd) : nullptr;
+    a.ws_conv = pl.chunked ? static_cast<void*>(ws + pl.off_conv) : nullptr;
+    a.dev_status = dev_status;
+    if (a.n_chunks_bound > 65535) return MDRAFT_ERR_UNSUPPORTED;
+    cudaError_t e = launch_prefill(a, act, pl.chunked, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MDRAFT_OK : MDRAFT_ERR_CUDA;
+}
+
+int mdraft_tree_step(const mdraft_layer* layer, const mdraft_cache* cache, int32_t layer_index, const void* x, int64_t ldx,
+                     const void* z, int64_t ldz, const void* dt, int64_t lddt, const void* B, int64_t ldb, const void* C,
+                     int64_t ldc, void* out, int64_t ldo, int32_t n_nodes, const int32_t* parent_slot,
+                     const int32_t* node_slot, int32_t n_levels, const int32_t* level_offsets, int32_t* dev_status,
+                     void* stream) {
+    int rc = check_layer(layer);
+    if (rc) return rc;
+    if ((rc = check_cache(cache, layer->d_inner, layer->act, layer_index))) return rc;
+    if (n_nodes < 0 || n_levels < 0) return MDRAFT_ERR_INVALID_ARG;
+    if (n_nodes == 0) return MDRAFT_OK;
+    if (!parent_slot || !node_slot) return MDRAFT_ERR_INVALID_ARG;
+    if (!level_offsets && n_levels > 1) return MDRAFT_ERR_INVALID_ARG;
+    if (level_offsets) {
+        if (n_levels < 1 || level_offsets[0] != 0 || level_offsets[n_levels] != n_nodes) return MDRAFT_ERR_INVALID_ARG;
+        for (int l = 0; l < n_levels; ++l)
+            if (level_offsets[l + 1] < level_offsets[l]) return MDRAFT_ERR_INVALID_ARG;
+    }
+    const bool conv_only = layer->flags & MDRAFT_CONV_ONLY;
+    const int D = layer->d_inner, act = layer->act;
+    if ((rc = check_matrix(x, ldx, D, act, true))) return rc;
+    if ((rc = check_matrix(out, ldo, D, act, true))) return rc;
+    if ((rc = check_matrix(z, ldz, D, act, !conv_only))) return rc;
+    if ((rc = check_matrix(dt, lddt, D, act, !conv_only))) return rc;
+    if ((rc = check_matrix(B, ldb, kN, act, !conv_only))) return rc;
+    if ((rc = check_matrix(C, ldc, kN, act, !conv_only))) return rc;
+
+    TreeArgs a;
+    a.L = layer_dev(layer);
+    a.pool = pool_dev(cache, act, layer_index);
+    a.x = x; a.z = z; a.dt = dt; a.B = B; a.C = C; a.out = out;
+    a.ldx = ldx; a.ldz = ldz; a.lddt = lddt; a.ldb = ldb; a.ldc = ldc; a.ldo = ldo;
+    a.parent_slot = parent_slot; a.node_slot = node_slot; a.dev_status = dev_status;
+    const int levels = level_offsets ? n_levels : 1;
+    for (int l = 0; l < levels; ++l) {
+        a.lvl_begin = level_offsets ? level_offsets[l] : 0;
+        a.lvl_end = level_offsets ? level_offsets[l + 1] : n_nodes;
+        if (launch_tree_step(a, act, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MDRAFT_ERR_CUDA;
+    }
+    return MDRAFT_OK;
+}
+
+int mdraft_state_commit(const mdraft_cache* cache, int32_t d_inner, int32_t d_state, int32_t d_conv, int32_t act,
+                        int32_t n_commit, const int32_t* src_slot, const int32_t* dst_slot, int32_t* dev_status,
+                        void* stream) {
+    if (d_inner <= 0 || n_commit < 0) return MDRAFT_ERR_INVALID_ARG;
+    if (d_state != kN || d_conv != kW || (d_inner % 8) != 0 || (act != MDRAFT_F32 && act != MDRAFT_BF16)) return MDRAFT_ERR_UNSUPPORTED;
+    int rc = check_cache(cache, d_inner, act, 0);
+    if (rc) return rc;
+    if (n_commit == 0) return MDRAFT_OK;
+    if (!src_slot || !dst_slot) return MDRAFT_ERR_INVALID_ARG;
+    const int64_t es = (int64_t)elem_size(act);
+    CommitArgs a;
+    a.ssm = reinterpret_cast<char*>(cache->ssm);
+    a.conv = static_cast<char*>(cache->conv);
+    a.ssm_layer_bytes = cache->ssm_layer_stride * 4; a.ssm_slot_bytes_stride = cache->ssm_slot_stride * 4;
+    a.conv_layer_bytes = cache->conv_layer_stride * es; a.conv_slot_bytes_stride = cache->conv_slot_stride * es;
+    a.ssm_bytes = (int64_t)d_inner * kN * 4; a.conv_bytes = (int64_t)(kW - 1) * d_inner * es;
+    a.n_layers = cache->n_layers; a.n_slots = cache->n_slots; a.dev_status = dev_status;
+    if (a.n_layers > 65535) return MDRAFT_ERR_UNSUPPORTED;
+    for (int off = 0; off < n_commit; off += 65535) {
+        a.n_commit = n_commit - off < 65535 ? n_commit - off : 65535;
+        a.src_slot = src_slot + off; a.dst_slot = dst_slot + off;
+        if (launch_commit(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MDRAFT_ERR_CUDA;
+    }
+    return MDRAFT_OK;
+}
+
+int mdraft_classify_A(const float* A, int32_t d_inner, int32_t d_state, int32_t* scratch, int32_t* is_powers,
+                      int32_t* is_nonpositive, void* stream) {
+    if (!A || !scratch || !is_powers || d_inner <= 0 || d_state <= 0) return MDRAFT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(scratch, 0, 2 * sizeof(int32_t), st) != cudaSuccess) return MDRAFT_ERR_CUDA;
+    const int n = d_inner * d_state;
+    classify_A_kernel<<<(n + 255) / 256, 256, 0, st>>>(A, d_inner, d_state, scratch);
+    int32_t host[2] = {1, 1};
+    if (cudaMemcpyAsync(host, scratch, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MDRAFT_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MDRAFT_ERR_CUDA;
+    *is_powers = host[0] == 0;
+    if (is_nonpositive) *is_nonpositive = host[1] == 0;
+    return MDRAFT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,119 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU, exports every function the header declares,
+and rejects bad arguments on the host before anything is launched (no GPU needed: no launch happens)."""
+
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2506_01206_b200.build import build_library
+    from paper_2506_01206_b200 import binding
+    build_library()
+    return binding.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "mdraft.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mdraft_[a-zA-Z0-9_]+)\s*\(", text)))
+
+
+def test_header_and_library_agree(lib):
+    from paper_2506_01206_b200 import binding
+    names = declared_functions()
+    assert "mdraft_conv_scan_prefill" in names and "mdraft_tree_step" in names and "mdraft_state_commit" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in include/mdraft.h but not exported"
+    assert sorted(binding.EXPORTS) == names, "the Python binding must expose exactly the declared entry points"
+    assert lib.mdraft_version() >= 100
+    assert lib.mdraft_status_string(0) == b"ok"
+    assert b"16 bytes" in lib.mdraft_status_string(-3)
+
+
+def _layer(binding, **kw):
+    base = dict(d_inner=64, d_state=16, d_conv=4, act=0, flags=1, reserved=0, A=0x1000, D=0, conv_w=0x2000, conv_b=0, dt_bias=0)
+    base.update(kw)
+    return binding._Layer(*[base[k] for k in ("d_inner", "d_state", "d_conv", "act", "flags", "reserved", "A", "D", "conv_w", "conv_b", "dt_bias")])
+
+
+def _cache(binding, **kw):
+    base = dict(ssm=0x10000, ssm_layer_stride=4 * 1024, ssm_slot_stride=1024, conv=0x20000, conv_layer_stride=4 * 192,
+                conv_slot_stride=192, n_layers=1, n_slots=4)
+    base.update(kw)
+    return binding._Cache(*[base[k] for k in ("ssm", "ssm_layer_stride", "ssm_slot_stride", "conv", "conv_layer_stride", "conv_slot_stride", "n_layers", "n_slots")])
+
+
+def _prefill(lib, binding, layer, cache, **kw):
+    a = dict(x=0x100000, ldx=64, z=0x200000, ldz=64, dt=0x300000, lddt=64, B=0x400000, ldb=16, C=0x500000, ldc=16,
+             out=0x600000, ldo=64, T=8, n_seq=1, max_seqlen=8, cu=0x700000, init=None, final=None, ws=None, ws_bytes=0, opts=None)
+    a.update(kw)
+    return lib.mdraft_conv_scan_prefill(C.byref(layer), C.byref(cache) if cache is not None else None, 0,
+                                        a["x"], a["ldx"], a["z"], a["ldz"], a["dt"], a["lddt"], a["B"], a["ldb"], a["C"], a["ldc"],
+                                        a["out"], a["ldo"], a["T"], a["n_seq"], a["max_seqlen"], a["cu"], a["init"], a["final"],
+                                        a["ws"], a["ws_bytes"], a["opts"], None, None)
+
+
+def test_host_side_argument_checks(lib):
+    from paper_2506_01206_b200 import binding
+    INVALID, UNSUPPORTED, MISALIGNED, WORKSPACE = -1, -2, -3, -4
+    ok_layer, ok_cache = _layer(binding), _cache(binding)
+    assert _prefill(lib, binding, _layer(binding, d_state=8), ok_cache) == UNSUPPORTED
+    assert _prefill(lib, binding, _layer(binding, d_conv=3), ok_cache) == UNSUPPORTED
+    assert _prefill(lib, binding, _layer(binding, d_inner=60), ok_cache) == UNSUPPORTED
+    assert _prefill(lib, binding, _layer(binding, act=7), ok_cache) == UNSUPPORTED
+    assert _prefill(lib, binding, _layer(binding, A=0), ok_cache) == INVALID
+    assert _prefill(lib, binding, _layer(binding, flags=2 | 4), ok_cache) == INVALID
+    assert _prefill(lib, binding, ok_layer, ok_cache, x=None) == INVALID
+    assert _prefill(lib, binding, ok_layer, ok_cache, cu=None) == INVALID
+    assert _prefill(lib, binding, ok_layer, ok_cache, ldx=32) == INVALID          # stride shorter than a row
+    assert _prefill(lib, binding, ok_layer, ok_cache, x=0x100004) == MISALIGNED
+    assert _prefill(lib, binding, ok_layer, ok_cache, ldb=18) == MISALIGNED       # 72-byte rows
+    assert _prefill(lib, binding, ok_layer, ok_cache, T=-1) == INVALID
+    assert _prefill(lib, binding, ok_layer, None, final=0x800000) == INVALID      # slots named but no pool
+    assert _prefill(lib, binding, ok_layer, _cache(binding, ssm_slot_stride=1000)) == INVALID
+    assert _prefill(lib, binding, ok_layer, _cache(binding, conv_slot_stride=194)) == MISALIGNED
+    # chunked plan without a workspace
+    opts = binding._PrefillOpts(); opts.chunk_len = 4
+    assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(opts)) == WORKSPACE
+    need = lib.mdraft_prefill_workspace_bytes(C.byref(ok_layer), 8, 1, 8, C.byref(opts))
+    assert need > 0 and need % 256 == 0
+    assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(opts), ws=0x900000, ws_bytes=need - 1) == WORKSPACE
+    assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(opts), ws=0x900010, ws_bytes=need) == MISALIGNED
+    bad = binding._PrefillOpts(); bad.chunk_len = 8; bad.reserved[3] = 1
+    assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(bad)) == INVALID
+    # nothing to do is fine and launches nothing
+    assert _prefill(lib, binding, ok_layer, ok_cache, n_seq=0, T=0, cu=None) == 0
+
+    def tree(layer=ok_layer, cache=ok_cache, n=4, parent=0xA00000, node=0xB00000, n_levels=1, levels=None, x=0x100000):
+        return lib.mdraft_tree_step(C.byref(layer), C.byref(cache) if cache is not None else None, 0, x, 64, 0x200000, 64,
+                                    0x300000, 64, 0x400000, 16, 0x500000, 16, 0x600000, 64, n, parent, node, n_levels, levels, None, None)
+
+    assert tree(cache=None) == INVALID
+    assert tree(parent=None) == INVALID
+    assert tree(n=0) == 0
+    assert tree(n_levels=2) == INVALID                                  # several levels need their offsets
+    assert tree(n_levels=2, levels=(C.c_int32 * 3)(0, 3, 5)) == INVALID     # must end at n_nodes
+    assert tree(n_levels=2, levels=(C.c_int32 * 3)(0, 5, 4)) == INVALID     # must not decrease
+    assert tree(layer=_layer(binding, d_state=32)) == UNSUPPORTED
+    assert tree(x=0x100002) == MISALIGNED
+
+    def commit(cache=ok_cache, d_inner=64, n=2, src=0xA00000, dst=0xB00000, act=0, d_state=16):
+        return lib.mdraft_state_commit(C.byref(cache) if cache is not None else None, d_inner, d_state, 4, act, n, src, dst, None, None)
+
+    assert commit(cache=None) == INVALID
+    assert commit(src=None) == INVALID
+    assert commit(n=0) == 0
+    assert commit(d_state=4) == UNSUPPORTED
+    assert commit(cache=_cache(binding, ssm_slot_stride=1026)) == MISALIGNED
+
+
+def test_missing_library_is_a_loud_error(tmp_path):
+    from paper_2506_01206_b200 import binding
+    with pytest.raises(ImportError):
+        binding.load_library(str(tmp_path / "nope.so"))
