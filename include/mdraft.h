@@ -111,10 +111,12 @@ typedef struct {
     int32_t n_layers, n_slots;
 } mdraft_cache;
 
-/* Optional tuning for the prefill; pass NULL for the defaults. */
+/* Optional tuning and profiling hooks for the prefill; pass NULL for the defaults. */
 typedef struct {
     int32_t chunk_len;      /* tokens per scan chunk; 0 = chosen from the problem size; otherwise >= 4   */
-    int32_t reserved[7];    /* must be 0 */
+    int32_t reserved[3];    /* must be 0 */
+    void *event_after_chunk_state;  /* cudaEvent_t or NULL: recorded on `stream` after the chunk-summary kernel  */
+    void *event_after_carry_scan;   /* cudaEvent_t or NULL: recorded after the carry scan, before the main scan  */
 } mdraft_prefill_opts;
 
 /*

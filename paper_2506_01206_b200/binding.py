@@ -49,7 +49,8 @@ class _Cache(C.Structure):
 
 
 class _PrefillOpts(C.Structure):
-    _fields_ = [("chunk_len", C.c_int32), ("reserved", C.c_int32 * 7)]
+    _fields_ = [("chunk_len", C.c_int32), ("reserved", C.c_int32 * 3),
+                ("event_after_chunk_state", C.c_void_p), ("event_after_carry_scan", C.c_void_p)]
 
 
 _lib = None
@@ -178,11 +179,14 @@ class StateCache:
         return self.ssm.numel() * 4 + self.conv.numel() * self.conv.element_size()
 
 
-def _opts(chunk_len: int):
-    if not chunk_len:
+def _opts(chunk_len: int, phase_events=None):
+    if not chunk_len and phase_events is None:
         return None
     o = _PrefillOpts()
     o.chunk_len = int(chunk_len)
+    if phase_events is not None:  # two torch.cuda.Event objects (already created with enable_timing=True)
+        o.event_after_chunk_state = phase_events[0].cuda_event
+        o.event_after_carry_scan = phase_events[1].cuda_event
     return C.byref(o)
 
 
@@ -196,7 +200,8 @@ def mdraft_conv_scan_prefill(layer: Layer, cache: Optional[StateCache], layer_in
                              x, z, dt, B, Cm, out, cu_seqlens: torch.Tensor, max_seqlen: int,
                              init_slot: Optional[torch.Tensor] = None, final_slot: Optional[torch.Tensor] = None,
                              workspace: Optional[torch.Tensor] = None, chunk_len: int = 0,
-                             dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None) -> None:
+                             dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None,
+                             phase_events=None) -> None:
     lib = load_library()
     cl = layer.c(flags)
     cc = cache.c() if cache is not None else None
@@ -213,7 +218,7 @@ def mdraft_conv_scan_prefill(layer: Layer, cache: Optional[StateCache], layer_in
     rc = lib.mdraft_conv_scan_prefill(C.byref(cl), C.byref(cc) if cc is not None else None, int(layer_index),
                                       px, ldx, pz, ldz, pdt, lddt, pB, ldb, pC, ldc, po, ldo,
                                       T, n_seq, int(max_seqlen), _ptr(cu_seqlens), _ptr(init_slot), _ptr(final_slot),
-                                      ws_ptr, ws_bytes, _opts(chunk_len), _ptr(dev_status), _stream_ptr(stream))
+                                      ws_ptr, ws_bytes, _opts(chunk_len, phase_events), _ptr(dev_status), _stream_ptr(stream))
     if rc != 0:
         raise MdraftError(rc, "mdraft_conv_scan_prefill")
 

@@ -146,7 +146,7 @@ int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cach
     if (total_tokens < 0 || n_seq < 0 || max_seqlen < 0) return MDRAFT_ERR_INVALID_ARG;
     if (opts) {
         if (opts->chunk_len < 0) return MDRAFT_ERR_INVALID_ARG;
-        for (int i = 0; i < 7; ++i)
+        for (int i = 0; i < 3; ++i)
             if (opts->reserved[i]) return MDRAFT_ERR_INVALID_ARG;
     }
     const bool needs_pool = init_slot || final_slot;
@@ -189,6 +189,8 @@ int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cach
     a.ws_conv = pl.chunked ? static_cast<void*>(ws + pl.off_conv) : nullptr;
     a.dev_status = dev_status;
     if (a.n_chunks_bound > 65535) return MDRAFT_ERR_UNSUPPORTED;
+    a.ev_state = opts ? static_cast<cudaEvent_t>(opts->event_after_chunk_state) : nullptr;
+    a.ev_carry = opts ? static_cast<cudaEvent_t>(opts->event_after_carry_scan) : nullptr;
     cudaError_t e = launch_prefill(a, act, pl.chunked, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? MDRAFT_OK : MDRAFT_ERR_CUDA;
 }

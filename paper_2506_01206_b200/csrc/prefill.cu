@@ -429,10 +429,15 @@ cudaError_t launch_typed(const PrefillArgs& p, bool chunked, cudaStream_t st) {
     const bool recur = !(p.L.flags & MDRAFT_CONV_ONLY);
     if (chunked) {
         chunk_state_kernel<AT, kPow><<<grid, kPrefillThreads, 0, st>>>(p);
+        if (p.ev_state) cudaEventRecord(p.ev_state, st);
         if (recur) {
             dim3 g2((D * kN + 31) / 32, p.n_seq);
             carry_scan_kernel<<<g2, 1024, 0, st>>>(p);
         }
+        if (p.ev_carry) cudaEventRecord(p.ev_carry, st);
+    } else {
+        if (p.ev_state) cudaEventRecord(p.ev_state, st);
+        if (p.ev_carry) cudaEventRecord(p.ev_carry, st);
     }
     chunk_scan_kernel<AT, kPow><<<grid, kPrefillThreads, 0, st>>>(p);
     return cudaGetLastError();

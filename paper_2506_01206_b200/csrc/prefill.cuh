@@ -19,6 +19,7 @@ struct PrefillArgs {
     float* ws_sd;   // [n_chunks_bound][D]    sum of Delta per chunk
     void* ws_conv;  // [n_seq][W-1][D]        starting conv windows (activation type)
     int32_t* dev_status;
+    cudaEvent_t ev_state, ev_carry;  // optional profiling events (host side only)
 };
 
 cudaError_t launch_prefill(const PrefillArgs& p, int act, bool chunked, cudaStream_t st);
