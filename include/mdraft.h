@@ -151,6 +151,38 @@ int mdraft_conv_scan_prefill(const mdraft_layer *layer, const mdraft_cache *cach
                              int32_t *dev_status, void *stream);
 
 /*
+ * The same prefill for callers that cannot allocate device memory.  No counterpart in the paper: this is a
+ * deployment variant of mdraft_conv_scan_prefill.  Some hosts of this library must never call cudaMalloc or a
+ * framework allocator once they are running: a serving loop whose memory pool was carved up at start-up, code
+ * that runs inside someone else's stream capture, a plug-in that is handed pointers but owns no allocator.
+ * They have nowhere to get the chunk workspace from, so this entry point brings its own: a fixed array of
+ * MDRAFT_NOALLOC_SCRATCH_BYTES inside the library image (every GPU that loads the library holds those bytes
+ * until the process exits).  Inputs, outputs and the state pool are still the caller's.
+ *
+ * Arguments and results are those of mdraft_conv_scan_prefill without `workspace` / `workspace_bytes`; the output
+ * is the same, bit for bit, as that call given a workspace of its own.
+ *   - A problem whose workspace (mdraft_prefill_workspace_bytes) exceeds MDRAFT_NOALLOC_SCRATCH_BYTES returns
+ *     MDRAFT_ERR_WORKSPACE before anything is launched: shorten the call (encode the context in pieces through
+ *     init_slot / final_slot) or use the entry point above with your own buffer.
+ *   - The first call on each device looks up the array's device address (the device must be current); make that
+ *     first call outside any stream capture.  Later calls do no set-up.
+ *   - Nothing is allocated or freed, here or in anything this calls.
+ *   - All calls on a device share the one array.  It holds whatever the previous call left; the prefill writes
+ *     every scratch word before reading it, so nothing needs clearing.  Two calls that may run at the same time
+ *     on one GPU (different streams, or different host threads) would overwrite each other's scratch: keep them
+ *     on one stream or otherwise ordered.
+ */
+#define MDRAFT_NOALLOC_SCRATCH_BYTES (8u << 20)
+
+int mdraft_conv_scan_prefill_noalloc(const mdraft_layer *layer, const mdraft_cache *cache, int32_t layer_index,
+                                     const void *x, int64_t ldx, const void *z, int64_t ldz, const void *dt, int64_t lddt,
+                                     const void *B, int64_t ldb, const void *C, int64_t ldc,
+                                     void *out, int64_t ldo,
+                                     int32_t total_tokens, int32_t n_seq, int32_t max_seqlen,
+                                     const int32_t *cu_seqlens, const int32_t *init_slot, const int32_t *final_slot,
+                                     const mdraft_prefill_opts *opts, int32_t *dev_status, void *stream);
+
+/*
  * Draft-tree step: one token for each of n_nodes nodes (of any number of
  * sequences) in one launch per tree level.  Node i reads the conv window and
  * SSM state in slot parent_slot[i], applies one step of the recurrence with its

@@ -24,7 +24,7 @@ MDRAFT_DT_SOFTPLUS, MDRAFT_PRECONV, MDRAFT_CONV_ONLY, MDRAFT_A_POWERS = 1, 2, 4,
 MDRAFT_DEV_BAD_SLOT, MDRAFT_DEV_BAD_SEQLENS, MDRAFT_DEV_WAIT_EXPIRED = 1, 2, 4
 
 EXPORTS = (
-    "mdraft_prefill_workspace_bytes", "mdraft_conv_scan_prefill", "mdraft_tree_step",
+    "mdraft_prefill_workspace_bytes", "mdraft_conv_scan_prefill", "mdraft_conv_scan_prefill_noalloc", "mdraft_tree_step",
     "mdraft_state_commit", "mdraft_classify_A", "mdraft_status_string", "mdraft_version",
 )
 
@@ -77,6 +77,10 @@ def load_library(path: Optional[str] = None):
     lib.mdraft_conv_scan_prefill.argtypes = [C.POINTER(_Layer), C.POINTER(_Cache), i32,
                                              vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                              i32, i32, i32, vp, vp, vp, vp, C.c_size_t, C.POINTER(_PrefillOpts), vp, vp]
+    lib.mdraft_conv_scan_prefill_noalloc.restype = C.c_int
+    lib.mdraft_conv_scan_prefill_noalloc.argtypes = [C.POINTER(_Layer), C.POINTER(_Cache), i32,
+                                                     vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
+                                                     i32, i32, i32, vp, vp, vp, C.POINTER(_PrefillOpts), vp, vp]
     lib.mdraft_tree_step.restype = C.c_int
     lib.mdraft_tree_step.argtypes = [C.POINTER(_Layer), C.POINTER(_Cache), i32,
                                      vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
@@ -221,6 +225,37 @@ def mdraft_conv_scan_prefill(layer: Layer, cache: Optional[StateCache], layer_in
                                       ws_ptr, ws_bytes, _opts(chunk_len, phase_events), _ptr(dev_status), _stream_ptr(stream))
     if rc != 0:
         raise MdraftError(rc, "mdraft_conv_scan_prefill")
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def mdraft_conv_scan_prefill_noalloc(layer: Layer, cache: Optional[StateCache], layer_index: int,
+                                     x, z, dt, B, Cm, out, cu_seqlens: torch.Tensor, max_seqlen: int,
+                                     init_slot: Optional[torch.Tensor] = None, final_slot: Optional[torch.Tensor] = None,
+                                     chunk_len: int = 0, dev_status: Optional[torch.Tensor] = None, stream=None,
+                                     flags: Optional[int] = None) -> None:
+    """Prefill without a caller workspace: the library's own fixed scratch array is used (see the header for
+    who needs this and for the sharing rules).  Raises MdraftError(MDRAFT_ERR_WORKSPACE) when the problem needs
+    more than NOALLOC_SCRATCH_BYTES of scratch."""
+    lib = load_library()
+    cl = layer.c(flags)
+    cc = cache.c() if cache is not None else None
+    px, ldx = _mat(x, "x"); pz, ldz = _mat(z, "z"); pdt, lddt = _mat(dt, "dt")
+    pB, ldb = _mat(B, "B"); pC, ldc = _mat(Cm, "C"); po, ldo = _mat(out, "out")
+    T = int(x.shape[0])
+    n_seq = int(cu_seqlens.numel()) - 1
+    if cu_seqlens.dtype != torch.int32:
+        raise TypeError("cu_seqlens must be int32")
+    for t, nm in ((init_slot, "init_slot"), (final_slot, "final_slot")):
+        if t is not None and (t.dtype != torch.int32 or t.numel() != n_seq):
+            raise TypeError(f"{nm} must be int32 with one entry per sequence")
+    rc = lib.mdraft_conv_scan_prefill_noalloc(C.byref(cl), C.byref(cc) if cc is not None else None, int(layer_index),
+                                              px, ldx, pz, ldz, pdt, lddt, pB, ldb, pC, ldc, po, ldo,
+                                              T, n_seq, int(max_seqlen), _ptr(cu_seqlens), _ptr(init_slot), _ptr(final_slot),
+                                              _opts(chunk_len), _ptr(dev_status), _stream_ptr(stream))
+    if rc != 0:
+        raise MdraftError(rc, "mdraft_conv_scan_prefill_noalloc")
 
 
 def mdraft_tree_step(layer: Layer, cache: StateCache, layer_index: int, x, z, dt, B, Cm, out,
