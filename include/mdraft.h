@@ -122,8 +122,9 @@ typedef struct {
 /*
  * Context encode ("prefill"): conv1d+SiLU, Delta activation, S6 scan and gate
  * over packed sequences, in parallel over channels and over chunks of tokens
- * whose (decay, input) summaries are combined by a prefix scan (the recurrence
- * is first-order linear, so chunks compose associatively).  Paper Section 3.1
+ * whose (decay, input) summaries are combined by a prefix scan into each chunk's
+ * incoming state (the recurrence is first-order linear, so chunks compose
+ * associatively).  Paper Section 3.1
  * (drafter encode) and Fig. 1a.
  *
  *   x, z, dt : (T, D) activations, strides ldx, ldz, lddt           [read]

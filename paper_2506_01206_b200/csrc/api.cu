@@ -1,5 +1,8 @@
 // C ABI of the library: argument checks, launch planning, dispatch.  No allocation, no global state.
+#include <cudaTypedefs.h>
 #include <limits.h>
+
+#include <string.h>
 
 #include "commit.cuh"
 #include "common.cuh"
@@ -68,10 +71,14 @@ struct PrefillPlan {
     int chunk_len;       // tokens per chunk (INT_MAX/2 when every sequence is one chunk)
     int n_chunks_bound;  // upper bound on the number of chunks
     bool chunked;
-    size_t off_h, off_sd, off_conv, bytes;
+    size_t off_q, off_sd, off_h0, off_conv, bytes;
 };
 
-// Chunk length: split the token axis only as far as needed to give every SM a few blocks.
+// Chunk length: split the token axis until every SM holds kBlocksPerSm blocks of kPrefillThreads channels (one
+// resident wave, no tail), but never into chunks shorter than kMinChunk tokens (per-chunk set-up would dominate) nor
+// longer than kMaxChunk (a batch of uneven sequences then still balances across SMs).
+constexpr int kBlocksPerSm = 4, kMinChunk = 32, kMaxChunk = 1024;
+
 PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen, const mdraft_prefill_opts* opts) {
     PrefillPlan pl;
     int Lc;
@@ -79,27 +86,59 @@ PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen
         Lc = opts->chunk_len < 4 ? 4 : opts->chunk_len;
     } else {
         const int ch_blocks = (L->d_inner + kPrefillThreads - 1) / kPrefillThreads;
-        const int want = (kSmCount * 4 + ch_blocks - 1) / ch_blocks;
+        int want = kSmCount * kBlocksPerSm / ch_blocks;
+        if (want < 1) want = 1;
         Lc = (T + want - 1) / want;
-        if (Lc < 64) Lc = 64;
-        Lc = (Lc + 31) / 32 * 32;
+        if (Lc < kMinChunk) Lc = kMinChunk;
+        if (Lc > kMaxChunk) Lc = kMaxChunk;
     }
     pl.chunked = Lc < max_seqlen;
     if (!pl.chunked) {
         pl.chunk_len = INT_MAX / 2;
         pl.n_chunks_bound = n_seq;
-        pl.off_h = pl.off_sd = pl.off_conv = 0;
+        pl.off_q = pl.off_sd = pl.off_h0 = pl.off_conv = 0;
         pl.bytes = 0;
         return pl;
     }
     pl.chunk_len = Lc;
     pl.n_chunks_bound = n_seq + T / Lc;
     const size_t D = (size_t)L->d_inner;
-    pl.off_h = 0;
-    pl.off_sd = align_up(pl.off_h + (size_t)pl.n_chunks_bound * D * kN * sizeof(float), 256);
-    pl.off_conv = align_up(pl.off_sd + (size_t)pl.n_chunks_bound * D * sizeof(float), 256);
+    pl.off_q = 0;
+    pl.off_sd = align_up(pl.off_q + (size_t)pl.n_chunks_bound * D * kN * sizeof(float), 256);
+    pl.off_h0 = align_up(pl.off_sd + (size_t)pl.n_chunks_bound * D * sizeof(float), 256);
+    pl.off_conv = align_up(pl.off_h0 + (size_t)n_seq * D * kN * sizeof(float), 256);
     pl.bytes = align_up(pl.off_conv + (size_t)n_seq * (kW - 1) * D * elem_size(L->act), 256);
     return pl;
+}
+
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library has no link-time dependency on the
+// driver (it can then be loaded, and its host-side checks exercised, on a machine without one).
+PFN_cuTensorMapEncodeTiled tensor_map_encoder() {
+    static PFN_cuTensorMapEncodeTiled fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) f = nullptr;
+        return reinterpret_cast<PFN_cuTensorMapEncodeTiled>(f);
+    }();
+    return fn;
+}
+
+// Descriptor of a (rows x cols) row-major activation matrix with row stride ld, read in boxes of box_cols x tile rows.
+bool encode_matrix(CUtensorMap* m, const void* base, int act, int64_t rows, int64_t cols, int64_t ld, int box_cols) {
+    PFN_cuTensorMapEncodeTiled enc = tensor_map_encoder();
+    if (!enc) return false;
+    if (!base) {  // tensor not used by this mode: leave a recognisable empty descriptor
+        memset(m, 0, sizeof(*m));
+        return true;
+    }
+    const cuuint64_t es = elem_size(act);
+    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)ld * es};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)(kPrefillTileRowBytes / es)};
+    cuuint32_t estride[2] = {1, 1};
+    return enc(m, act == MDRAFT_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
+               gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 __global__ void classify_A_kernel(const float* A, int D, int N, int32_t* res) {
@@ -184,14 +223,22 @@ int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cach
     a.T = total_tokens; a.n_seq = n_seq; a.chunk_len = pl.chunk_len; a.n_chunks_bound = pl.n_chunks_bound;
     a.cu = cu_seqlens; a.init_slot = init_slot; a.final_slot = final_slot;
     char* ws = static_cast<char*>(workspace);
-    a.ws_h = pl.chunked ? reinterpret_cast<float*>(ws + pl.off_h) : nullptr;
+    a.ws_q = pl.chunked ? reinterpret_cast<float*>(ws + pl.off_q) : nullptr;
     a.ws_sd = pl.chunked ? reinterpret_cast<float*>(ws + pl.off_sd) : nullptr;
+    a.ws_h0 = pl.chunked ? reinterpret_cast<float*>(ws + pl.off_h0) : nullptr;
     a.ws_conv = pl.chunked ? static_cast<void*>(ws + pl.off_conv) : nullptr;
     a.dev_status = dev_status;
     if (a.n_chunks_bound > 65535) return MDRAFT_ERR_UNSUPPORTED;
     a.ev_state = opts ? static_cast<cudaEvent_t>(opts->event_after_chunk_state) : nullptr;
     a.ev_carry = opts ? static_cast<cudaEvent_t>(opts->event_after_carry_scan) : nullptr;
-    cudaError_t e = launch_prefill(a, act, pl.chunked, static_cast<cudaStream_t>(stream));
+    PrefillMaps maps;  // with no tokens at all (only empty sequences) nothing is ever copied: empty descriptors
+    if (!encode_matrix(&maps.x, have_rows ? x : nullptr, act, total_tokens, D, ldx, kPrefillThreads) ||
+        !encode_matrix(&maps.dt, have_rows ? dt : nullptr, act, total_tokens, D, lddt, kPrefillThreads) ||
+        !encode_matrix(&maps.z, have_rows ? z : nullptr, act, total_tokens, D, ldz, kPrefillThreads) ||
+        !encode_matrix(&maps.B, have_rows ? B : nullptr, act, total_tokens, kN, ldb, kN) ||
+        !encode_matrix(&maps.C, have_rows ? C : nullptr, act, total_tokens, kN, ldc, kN))
+        return MDRAFT_ERR_CUDA;
+    cudaError_t e = launch_prefill(a, maps, act, pl.chunked, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? MDRAFT_OK : MDRAFT_ERR_CUDA;
 }
 

@@ -3,11 +3,26 @@
 // The recurrence h_t = a_t h_{t-1} + b_t is first-order linear, so a chunk of tokens acts on the incoming
 // state as h_out = P h_in + q with P = prod a_t = exp(A * sum Delta_t) and q = the chunk's result from a zero
 // state.  Three stream-ordered kernels, none of which waits on another block:
-//   1. chunk_state : every chunk but the last of a sequence computes (sum Delta, q) from a zero state.
-//   2. carry_scan  : per (channel, state) the (P, q) pairs of a sequence are combined in token order with a
-//                    warp-shuffle inclusive scan (lanes = chunks); the result is each chunk's incoming state.
-//   3. chunk_scan  : every chunk re-runs its tokens from the true incoming state and writes the outputs.
-// A sequence that fits one chunk skips 1 and 2.
+//   1. summary pass (chunk_kernel, kOut = false): every chunk but the last of a sequence computes (sum Delta, q)
+//      from a zero state; the first chunk of a split sequence also stashes the sequence's starting conv window.
+//   2. carry scan: per (channel, state) the (P, q) pairs of a sequence are combined in token order (eight groups
+//      of chunks folded side by side, group results exchanged through shared memory); entry c of the summary
+//      array is overwritten with the state after chunk c, and the starting state is stashed, so that the final
+//      state may later be written to the slot the starting state came from.
+//   3. output pass (chunk_kernel, kOut = true): every chunk starts from its incoming state, runs its tokens and
+//      writes the outputs; the last chunk stores the final state and conv window.
+// A call in which every sequence fits one chunk runs the output pass only.
+//
+// Data movement.  One thread owns one channel and keeps its 16 state entries in registers as 8 packed pairs
+// (fma.rn.f32x2 / mul.rn.f32x2: one instruction per two entries).  A block of 128 channels walks its chunk in
+// tiles of 16 (bf16) or 8 (fp32) tokens; the x / dt / z boxes (tile x 128 channels) and the B / C boxes of a tile
+// are brought into a ring of shared-memory stages by TMA (cp.async.bulk.tensor, one instruction per matrix and
+// tile, completion counted on an mbarrier), two tiles ahead of the arithmetic.  The block is warp-specialised: a fifth warp queues the copies,
+// widens each landed B / C tile to fp32 (read afterwards as 128-bit broadcasts) and hands it to the four
+// channel warps through a "ready" mbarrier; each channel warp releases a stage through an "empty" mbarrier
+// when it is done, so the channel warps never wait for one another.  Every wait on an mbarrier is bounded: if
+// it runs out, the warp raises MDRAFT_DEV_WAIT_EXPIRED and stops; the copy warp first gives the copies it still
+// has in flight a bounded chance to land (they target this block's shared memory).
 #include "common.cuh"
 #include "prefill.cuh"
 
@@ -15,8 +30,78 @@ namespace mdraft {
 
 namespace {
 
-constexpr int kTT = 32;  // tokens per shared-memory tile of B / C
+constexpr int kCB = kPrefillThreads;    // channels per block, one thread each
+constexpr int kBlockThreads = kCB + 32; // plus the copy warp
+constexpr int kStages = 3;              // shared-memory ring depth
+constexpr int kTileBytes = 4096;        // one staged x / dt / z tile: kTT rows of kCB activations
+constexpr int kBCBytes = 512;           // one staged B or C tile: kTT rows of 16 activations
+constexpr int kStageBytes = 3 * kTileBytes + 2 * kBCBytes;
+constexpr int kOffX = 0, kOffDt = kTileBytes, kOffZ = 2 * kTileBytes, kOffB = 3 * kTileBytes, kOffC = 3 * kTileBytes + kBCBytes;
+constexpr uint32_t kSpinLimit = 1u << 20;  // polls of one mbarrier before the block gives up
 
+template <typename AT> struct TileTokens { static constexpr int v = kPrefillTileRowBytes / (int)sizeof(AT); };  // 16 (bf16) or 8 (fp32)
+
+typedef unsigned long long u64;
+
+// ---------------------------------------------------------------- packed fp32 pairs
+__device__ __forceinline__ u64 pk(float lo, float hi) {
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpk(u64 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ float hi_of(u64 v) {
+    float lo, hi;
+    unpk(v, lo, hi);
+    return hi;
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ u64 mul2(u64 a, u64 b) {
+    u64 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// ---------------------------------------------------------------- mbarrier + bulk copy
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// One 2-D box of a matrix -> shared memory (TMA).  `col` times the element size must be a multiple of 16 bytes;
+// rows or columns of the box that fall outside the matrix arrive as zeros and still count towards the
+// transaction bytes.
+__device__ __forceinline__ void tma_box(void* dst, const CUtensorMap* map, int col, int row, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_u32(dst)),
+                 "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(row), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// ---------------------------------------------------------------- chunk bookkeeping
 struct ChunkInfo {
     int seq;     // sequence index, -1 if this chunk id is past the last chunk
     int k;       // chunk index within the sequence
@@ -99,37 +184,70 @@ __device__ void seq_chunks(const int32_t* cu, int n_seq, int T, int Lc, int s, i
 
 __device__ __forceinline__ int load_slot(const int32_t* slots, int s) { return slots ? __ldg(slots + s) : -1; }
 
-// ---------------------------------------------------------------------------------------------------
-// Per-channel running computation shared by chunk_state (kOut = false) and chunk_scan (kOut = true).
-template <typename AT, bool kPow, bool kOut>
+// ---------------------------------------------------------------- one channel's running computation
+template <typename AT, bool kPow, bool kOut, bool kFast>
 struct ChannelScan {
-    float h[kN];
-    float a2[kN];      // general A: A[d][n] * log2(e);   powers: only a2[0] is used
+    u64 h[kN / 2];        // state, entries (2k, 2k+1) packed
+    u64 a2[kN / 2];       // general A: A[d][n] * log2(e), packed;  structured A: only a20 is used
+    float a20;
     float w[kW];
-    float win[kW - 1]; // previous raw inputs, oldest first
+    float win[kW - 1];    // previous raw inputs, oldest first
     float cb, dtb, dsk, sum_delta;
     uint32_t flags;
 
     __device__ __forceinline__ void init(const LayerDev& L, int d) {
+        const float4* Ap = reinterpret_cast<const float4*>(L.A + (size_t)d * kN);
 #pragma unroll
-        for (int n = 0; n < kN; ++n) a2[n] = __ldg(L.A + (size_t)d * kN + n) * kLog2e;
-#pragma unroll
-        for (int k = 0; k < kW; ++k) w[k] = __ldg(L.conv_w + (size_t)d * kW + k);
+        for (int q = 0; q < kN / 4; ++q) {
+            float4 a = __ldg(Ap + q);
+            a2[2 * q] = pk(a.x * kLog2e, a.y * kLog2e);
+            a2[2 * q + 1] = pk(a.z * kLog2e, a.w * kLog2e);
+            if (q == 0) a20 = a.x * kLog2e;
+        }
+        float4 wv = __ldg(reinterpret_cast<const float4*>(L.conv_w + (size_t)d * kW));
+        w[0] = wv.x; w[1] = wv.y; w[2] = wv.z; w[3] = wv.w;
         cb = L.conv_b ? __ldg(L.conv_b + d) : 0.0f;
         dtb = L.dt_bias ? __ldg(L.dt_bias + d) : 0.0f;
         dsk = L.D ? __ldg(L.D + d) : 0.0f;
         sum_delta = 0.0f;
-        flags = L.flags;
+        flags = kFast ? (uint32_t)MDRAFT_DT_SOFTPLUS : L.flags;
+#pragma unroll
+        for (int k = 0; k < kN / 2; ++k) h[k] = pk(0.0f, 0.0f);
     }
 
-    // One token.  Bt / Ct point at 16 fp32 values in shared memory.  Returns out (kOut) or is unused.
+    // The 16 decays exp(A[d][n] * delta) as 8 packed pairs.
+    __device__ __forceinline__ void decays(float delta, u64 (&P)[kN / 2]) const {
+        if (kPow) {
+            const float r1 = ex2(delta * a20);
+            const float r2 = r1 * r1;
+            P[0] = pk(r1, r2);
+            P[1] = mul2(P[0], pk(r2, r2));
+            const float r4 = hi_of(P[1]);
+            const u64 R4 = pk(r4, r4);
+            P[2] = mul2(P[0], R4);
+            P[3] = mul2(P[1], R4);
+            const float r8 = hi_of(P[3]);
+            const u64 R8 = pk(r8, r8);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) P[4 + k] = mul2(P[k], R8);
+        } else {
+            const u64 dd = pk(delta, delta);
+#pragma unroll
+            for (int k = 0; k < kN / 2; ++k) {
+                float lo, hi;
+                unpk(mul2(dd, a2[k]), lo, hi);
+                P[k] = pk(ex2(lo), ex2(hi));
+            }
+        }
+    }
+
+    // One token.  Bt / Ct point at 16 fp32 values in shared memory.  Returns the output (kOut) or u (conv only).
     __device__ __forceinline__ float token(float xv, float zv, float dtv, const float* Bt, const float* Ct) {
         float u;
         if (flags & MDRAFT_PRECONV) {
             u = xv;
         } else {
-            float acc = cb;
-            acc = fmaf(w[0], win[0], acc);
+            float acc = fmaf(w[0], win[0], cb);
             acc = fmaf(w[1], win[1], acc);
             acc = fmaf(w[2], win[2], acc);
             acc = fmaf(w[3], xv, acc);
@@ -137,56 +255,35 @@ struct ChannelScan {
             u = silu(acc);
         }
         if (flags & MDRAFT_CONV_ONLY) return u;
-        float v = dtv + dtb;
-        float delta = (flags & MDRAFT_DT_SOFTPLUS) ? softplus(v) : v;
-        sum_delta += delta;
-        float du = delta * u;
-        float dA[kN];
-        if (kPow) {
-            float r1 = ex2(delta * a2[0]);
-            float r2 = r1 * r1, r4 = r2 * r2, r8 = r4 * r4;
-            dA[0] = r1; dA[1] = r2; dA[2] = r2 * r1; dA[3] = r4;
-            dA[4] = r4 * r1; dA[5] = r4 * r2; dA[6] = r4 * dA[2]; dA[7] = r8;
-#pragma unroll
-            for (int n = 0; n < 8; ++n) dA[8 + n] = r8 * dA[n];
-        } else {
-#pragma unroll
-            for (int n = 0; n < kN; ++n) dA[n] = ex2(delta * a2[n]);
-        }
-        float y0 = 0.0f, y1 = 0.0f;
+        const float v = dtv + dtb;
+        const float delta = (flags & MDRAFT_DT_SOFTPLUS) ? softplus(v) : v;
+        if (!kOut) sum_delta += delta;
+        const float du = delta * u;
+        u64 P[kN / 2];
+        decays(delta, P);
+        const u64 DU = pk(du, du);
+        u64 y0 = pk(0.0f, 0.0f), y1 = pk(0.0f, 0.0f);
+        const ulonglong2* B2 = reinterpret_cast<const ulonglong2*>(Bt);
+        const ulonglong2* C2 = reinterpret_cast<const ulonglong2*>(Ct);
 #pragma unroll
         for (int q = 0; q < kN / 4; ++q) {
-            float4 b4 = *reinterpret_cast<const float4*>(Bt + 4 * q);
-            float bb[4] = {b4.x, b4.y, b4.z, b4.w};
-            float cc[4] = {0.f, 0.f, 0.f, 0.f};
+            const ulonglong2 b = B2[q];
+            h[2 * q] = fma2(P[2 * q], h[2 * q], mul2(DU, b.x));
+            h[2 * q + 1] = fma2(P[2 * q + 1], h[2 * q + 1], mul2(DU, b.y));
             if (kOut) {
-                float4 c4 = *reinterpret_cast<const float4*>(Ct + 4 * q);
-                cc[0] = c4.x; cc[1] = c4.y; cc[2] = c4.z; cc[3] = c4.w;
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                int n = 4 * q + j;
-                h[n] = fmaf(dA[n], h[n], du * bb[j]);
-                if (kOut) {
-                    if (j & 1) y1 = fmaf(cc[j], h[n], y1); else y0 = fmaf(cc[j], h[n], y0);
-                }
+                const ulonglong2 c = C2[q];
+                y0 = fma2(c.x, h[2 * q], y0);
+                y1 = fma2(c.y, h[2 * q + 1], y1);
             }
         }
         if (!kOut) return 0.0f;
-        float y = fmaf(dsk, u, y0 + y1);
+        float ya, yb, yc, yd;
+        unpk(y0, ya, yb);
+        unpk(y1, yc, yd);
+        const float y = fmaf(dsk, u, (ya + yb) + (yc + yd));
         return y * silu(zv);
     }
 };
-
-template <typename AT>
-__device__ __forceinline__ void stage_bc(float (*sB)[kN], float (*sC)[kN], const AT* B, const AT* C, int64_t ldb, int64_t ldc,
-                                         int t, int rows, bool want_c) {
-    for (int i = threadIdx.x; i < rows * kN; i += blockDim.x) {
-        int r = i / kN, n = i % kN;
-        sB[r][n] = Act<AT>::load(B + (size_t)(t + r) * ldb + n);
-        if (want_c) sC[r][n] = Act<AT>::load(C + (size_t)(t + r) * ldc + n);
-    }
-}
 
 // Conv window at the start of a chunk: the W-1 rows before t0, taken from the sequence itself, or (chunk 0)
 // from `src_rows` = (W-1, D) activations, or zeros.
@@ -199,222 +296,243 @@ __device__ __forceinline__ void load_window(float* win, const AT* x, int64_t ldx
     }
 }
 
-// ---------------------------------------------------------------------------------------------------
-template <typename AT, bool kPow>
-__global__ void __launch_bounds__(kPrefillThreads) chunk_state_kernel(PrefillArgs p) {
-    __shared__ __align__(16) float sB[kTT][kN];
-    const int D = p.L.d_inner;
-    const int d = blockIdx.x * blockDim.x + threadIdx.x;
-    const bool live = d < D;
-    const int cidx = blockIdx.y;
-    ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, p.chunk_len, cidx);
-    if (ci.seq < 0 || ci.k == ci.nck - 1) return;  // the last chunk's summary is never used
-
-    const AT* x = static_cast<const AT*>(p.x);
-    const AT* dt = static_cast<const AT*>(p.dt);
-    const AT* B = static_cast<const AT*>(p.B);
-
-    ChannelScan<AT, kPow, false> cs;
-    if (live) {
-        cs.init(p.L, d);
-        const AT* rows = nullptr;
-        if (ci.k == 0) {
-            int slot = load_slot(p.init_slot, ci.seq);
-            if (slot >= 0 && slot < p.pool.n_slots) rows = static_cast<const AT*>(p.pool.conv) + (size_t)slot * p.pool.conv_slot_stride;
-        }
-        load_window<AT>(cs.win, x, p.ldx, d, ci.t0, ci.k, rows, D);
-        if (ci.k == 0) {  // keep the sequence's starting window where chunk_scan can read it even if the slot is overwritten
-            AT* stash = static_cast<AT*>(p.ws_conv) + (size_t)ci.seq * (kW - 1) * D;
-#pragma unroll
-            for (int j = 0; j < kW - 1; ++j) stash[(size_t)j * D + d] = Act<AT>::from_f32(cs.win[j]);
-        }
-#pragma unroll
-        for (int n = 0; n < kN; ++n) cs.h[n] = 0.0f;
-    }
-    if (p.L.flags & MDRAFT_CONV_ONLY) return;  // no recurrence: the stash was all this kernel had to do
-    for (int t = ci.t0; t < ci.t1; t += kTT) {
-        int rows = min(kTT, ci.t1 - t);
-        __syncthreads();
-        stage_bc<AT>(sB, sB, B, B, p.ldb, p.ldb, t, rows, false);
-        __syncthreads();
-        if (live) {
-#pragma unroll 4
-            for (int r = 0; r < rows; ++r) {
-                float xv = Act<AT>::load(x + (size_t)(t + r) * p.ldx + d);
-                float dtv = Act<AT>::load(dt + (size_t)(t + r) * p.lddt + d);
-                cs.token(xv, 0.0f, dtv, sB[r], sB[r]);
-            }
-        }
-    }
-    if (live) {
-        float4* dst = reinterpret_cast<float4*>(p.ws_h + ((size_t)cidx * D + d) * kN);
-#pragma unroll
-        for (int q = 0; q < kN / 4; ++q) dst[q] = make_float4(cs.h[4 * q], cs.h[4 * q + 1], cs.h[4 * q + 2], cs.h[4 * q + 3]);
-        p.ws_sd[(size_t)cidx * D + d] = cs.sum_delta;
-    }
+// One lane queues the copies of one tile: a box per matrix.  `mask`: bit 0 = dt, bit 1 = z, bit 2 = B, bit 3 = C
+// (x is always copied).  Every box is full size whatever part of it lies inside the matrix.
+__device__ __forceinline__ void issue_tile(unsigned char* stage, uint64_t* bar, const PrefillMaps& m, int t, int d0, uint32_t mask) {
+    const uint32_t n_wide = 1u + (mask & 1u) + ((mask >> 1) & 1u), n_bc = ((mask >> 2) & 1u) + ((mask >> 3) & 1u);
+    mbar_expect_tx(bar, n_wide * kTileBytes + n_bc * kBCBytes);
+    tma_box(stage + kOffX, &m.x, d0, t, bar);
+    if (mask & 1u) tma_box(stage + kOffDt, &m.dt, d0, t, bar);
+    if (mask & 2u) tma_box(stage + kOffZ, &m.z, d0, t, bar);
+    if (mask & 4u) tma_box(stage + kOffB, &m.B, 0, t, bar);
+    if (mask & 8u) tma_box(stage + kOffC, &m.C, 0, t, bar);
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Block = 32 warps.  Tile = 32 consecutive (d, n) elements x 32 consecutive chunks of one sequence.
-// Load: warp j reads chunk j's 32 elements (one 128-byte line).  Scan: warp j owns element j, lanes = chunks,
-// Hillis-Steele inclusive scan of (P, q) under (P2,q2)o(P1,q1) = (P1*P2, P2*q1 + q2).  The incoming state of
-// chunk k+1 is stored where chunk k's summary was.
-__global__ void __launch_bounds__(1024) carry_scan_kernel(PrefillArgs p) {
-    __shared__ float sP[32][33];
-    __shared__ float sQ[32][33];
-    __shared__ float carry[32];
-    const unsigned full = 0xffffffffu;
-    const int D = p.L.d_inner;
-    const int E = D * kN;
-    const int lane = threadIdx.x & 31, wj = threadIdx.x >> 5;
-    const int e0 = blockIdx.x * 32;
-    const int s = blockIdx.y;
-    int first, nck;
-    seq_chunks(p.cu, p.n_seq, p.T, p.chunk_len, s, first, nck);
-    if (nck <= 1) return;
+template <typename AT, bool kPow, bool kOut, bool kFast>
+__global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs p, const __grid_constant__ PrefillMaps maps) {
+    constexpr int TT = TileTokens<AT>::v;
+    __shared__ __align__(128) unsigned char s_stage[kStages][kStageBytes];
+    __shared__ __align__(16) float sBf[kStages][TT][kN];
+    __shared__ __align__(16) float sCf[kStages][TT][kN];
+    __shared__ __align__(8) uint64_t bar_raw[kStages];    // copies of a tile have landed (transaction count)
+    __shared__ __align__(8) uint64_t bar_ready[kStages];  // ... and its B / C are widened: channel warps may start
+    __shared__ __align__(8) uint64_t bar_empty[kStages];  // all channel warps are done with the stage
 
-    if (wj == 0) {
-        int e = e0 + lane;
-        float h0 = 0.0f;
-        int slot = load_slot(p.init_slot, s);
-        if (e < E && slot >= 0 && slot < p.pool.n_slots) h0 = p.pool.ssm[(size_t)slot * p.pool.ssm_slot_stride + e];
-        carry[lane] = h0;
-    }
-    const int n_sum = nck - 1;  // summaries of chunks 0 .. nck-2
-    for (int b0 = 0; b0 < n_sum; b0 += 32) {
-        __syncthreads();
-        {
-            int k = b0 + wj, e = e0 + lane;
-            float P = 1.0f, q = 0.0f;
-            if (k < n_sum && e < E) {
-                size_t c = (size_t)(first + k);
-                q = p.ws_h[c * E + e];
-                float sd = p.ws_sd[c * D + e / kN];
-                P = ex2(__ldg(p.L.A + e) * kLog2e * sd);
-            }
-            sP[wj][lane] = P;
-            sQ[wj][lane] = q;
-        }
-        __syncthreads();
-        {
-            float P = sP[lane][wj], q = sQ[lane][wj];
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                float Pp = __shfl_up_sync(full, P, o);
-                float qp = __shfl_up_sync(full, q, o);
-                if (lane >= o) { q = fmaf(P, qp, q); P = P * Pp; }
-            }
-            float hin = fmaf(P, carry[wj], q);  // state after chunk b0+lane = incoming state of chunk b0+lane+1
-            sQ[lane][wj] = hin;
-            __syncwarp();
-            if (lane == 31) carry[wj] = hin;
-        }
-        __syncthreads();
-        {
-            int k = b0 + wj, e = e0 + lane;
-            if (k < n_sum && e < E) p.ws_h[(size_t)(first + k) * E + e] = sQ[wj][lane];
-        }
-    }
-}
-
-// ---------------------------------------------------------------------------------------------------
-template <typename AT, bool kPow>
-__global__ void __launch_bounds__(kPrefillThreads) chunk_scan_kernel(PrefillArgs p) {
-    __shared__ __align__(16) float sB[kTT][kN];
-    __shared__ __align__(16) float sC[kTT][kN];
     const int D = p.L.d_inner;
-    const int d = blockIdx.x * blockDim.x + threadIdx.x;
-    const bool live = d < D;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int d0 = blockIdx.x * kCB;
+    const int cols = min(kCB, D - d0);
+    const int d = d0 + tid;
+    const bool live = tid < cols;            // false for the copy warp (tid >= kCB) as well
+    const bool copy_warp = warp == kCB / 32;
     const int cidx = blockIdx.y;
+    const uint32_t flags = kFast ? (uint32_t)MDRAFT_DT_SOFTPLUS : p.L.flags;
+    const bool conv_only = flags & MDRAFT_CONV_ONLY, preconv = flags & MDRAFT_PRECONV;
 
-    // Sequences without tokens have no chunk: their final state is their starting state.
-    if (cidx == 0 && p.final_slot) {
-        for (int s = 0; s < p.n_seq; ++s) {
-            int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
-            bool bad = (lo < 0) || (hi < lo) || (hi > p.T);
-            if (bad && blockIdx.x == 0 && threadIdx.x == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);
-            if (bad || hi != lo) continue;
-            int fs = __ldg(p.final_slot + s), is = load_slot(p.init_slot, s);
-            if (fs < 0 || fs == is) continue;
-            if (fs >= p.pool.n_slots || is >= p.pool.n_slots) {
-                if (blockIdx.x == 0 && threadIdx.x == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
-                continue;
-            }
-            if (live) {
-                float* dh = p.pool.ssm + (size_t)fs * p.pool.ssm_slot_stride + (size_t)d * kN;
-                AT* dc = static_cast<AT*>(p.pool.conv) + (size_t)fs * p.pool.conv_slot_stride;
-                const float* sh = is >= 0 ? p.pool.ssm + (size_t)is * p.pool.ssm_slot_stride + (size_t)d * kN : nullptr;
-                const AT* sc = is >= 0 ? static_cast<const AT*>(p.pool.conv) + (size_t)is * p.pool.conv_slot_stride : nullptr;
-                for (int n = 0; n < kN; ++n) dh[n] = sh ? sh[n] : 0.0f;
-                for (int j = 0; j < kW - 1; ++j) dc[(size_t)j * D + d] = sc ? sc[(size_t)j * D + d] : Act<AT>::from_f32(0.0f);
-            }
+    if (tid == 0) {
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&bar_raw[s], 1);
+            mbar_init(&bar_ready[s], 1);
+            mbar_init(&bar_empty[s], kCB / 32);
         }
-    } else if (cidx == 0 && blockIdx.x == 0 && threadIdx.x < 32) {
-        for (int s = threadIdx.x; s < p.n_seq; s += 32) {
-            int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
-            if ((lo < 0) || (hi < lo) || (hi > p.T)) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (kOut) {
+        // Sequences without tokens have no chunk: their final state is their starting state.
+        if (cidx == 0 && p.final_slot) {
+            for (int s = 0; s < p.n_seq; ++s) {
+                int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
+                bool bad = (lo < 0) || (hi < lo) || (hi > p.T);
+                if (bad && blockIdx.x == 0 && tid == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);
+                if (bad || hi != lo) continue;
+                int fs = __ldg(p.final_slot + s), is = load_slot(p.init_slot, s);
+                if (fs < 0 || fs == is) continue;
+                if (fs >= p.pool.n_slots || is >= p.pool.n_slots) {
+                    if (blockIdx.x == 0 && tid == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+                    continue;
+                }
+                if (live) {
+                    float* dh = p.pool.ssm + (size_t)fs * p.pool.ssm_slot_stride + (size_t)d * kN;
+                    AT* dc = static_cast<AT*>(p.pool.conv) + (size_t)fs * p.pool.conv_slot_stride;
+                    const float* sh = is >= 0 ? p.pool.ssm + (size_t)is * p.pool.ssm_slot_stride + (size_t)d * kN : nullptr;
+                    const AT* sc = is >= 0 ? static_cast<const AT*>(p.pool.conv) + (size_t)is * p.pool.conv_slot_stride : nullptr;
+                    for (int n = 0; n < kN; ++n) dh[n] = sh ? sh[n] : 0.0f;
+                    for (int j = 0; j < kW - 1; ++j) dc[(size_t)j * D + d] = sc ? sc[(size_t)j * D + d] : Act<AT>::from_f32(0.0f);
+                }
+            }
+        } else if (cidx == 0 && blockIdx.x == 0 && tid < 32) {
+            for (int s = tid; s < p.n_seq; s += 32) {
+                int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
+                if ((lo < 0) || (hi < lo) || (hi > p.T)) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);
+            }
         }
     }
 
-    ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, p.chunk_len, cidx);
+    const ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, p.chunk_len, cidx);
     if (ci.seq < 0) return;
+    if (!kOut) {
+        // No summary is needed for an unsplit sequence or for a sequence's last chunk; in conv-only mode the only
+        // job left is the first chunk's stash of the starting window.
+        if (ci.nck == 1 || ci.k == ci.nck - 1) return;
+        if ((flags & MDRAFT_CONV_ONLY) && ci.k > 0) return;
+    }
 
-    const AT* x = static_cast<const AT*>(p.x);
-    const AT* z = static_cast<const AT*>(p.z);
-    const AT* dt = static_cast<const AT*>(p.dt);
-    const AT* B = static_cast<const AT*>(p.B);
-    const AT* C = static_cast<const AT*>(p.C);
-    AT* out = static_cast<AT*>(p.out);
-
-    int islot = load_slot(p.init_slot, ci.seq);
-    int fslot = load_slot(p.final_slot, ci.seq);
+    const int islot = load_slot(p.init_slot, ci.seq);
+    const int fslot = load_slot(p.final_slot, ci.seq);
     if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) {  // whole sequence becomes a no-op
-        if (threadIdx.x == 0 && blockIdx.x == 0 && ci.k == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+        if (kOut && tid == 0 && blockIdx.x == 0 && ci.k == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
         return;
     }
 
-    ChannelScan<AT, kPow, true> cs;
+    const AT* x = static_cast<const AT*>(p.x);
+    AT* out = static_cast<AT*>(p.out);
+
+    // In conv-only mode the summary pass computes nothing (it only stashes, below).
+    const bool compute = kOut || !conv_only;
+    const int ntiles = compute ? (ci.t1 - ci.t0 + TT - 1) / TT : 0;
+    uint32_t mask = 0;
+    if (!conv_only) mask = kOut ? 15u : 5u;  // summary pass: x, dt, B
+
+    const bool want_c = kOut && !conv_only;
+    if (copy_warp) {
+        // ---- copy warp: keep two tiles in flight, widen B / C of each landed tile, hand it over.
+        const int pre = min(kStages - 1, ntiles);
+        if (lane == 0)
+            for (int j = 0; j < pre; ++j) issue_tile(s_stage[j], &bar_raw[j], maps, ci.t0 + j * TT, d0, mask);
+        int landed = 0, queued = pre;  // tiles [landed, queued) are in flight
+        bool ok = true;
+        for (int j = 0; j < ntiles && ok; ++j) {
+            const int s = j % kStages;
+            ok = mbar_wait_bounded(&bar_raw[s], (uint32_t)(j / kStages) & 1u);
+            if (!ok) break;
+            landed = j + 1;
+            if (!conv_only) {
+                const int rows = min(TT, ci.t1 - (ci.t0 + j * TT));
+                const AT* rb = reinterpret_cast<const AT*>(s_stage[s] + kOffB);
+                const AT* rc = reinterpret_cast<const AT*>(s_stage[s] + kOffC);
+                for (int i = lane; i < rows * kN; i += 32) {
+                    (&sBf[s][0][0])[i] = Act<AT>::to_f32(rb[i]);
+                    if (want_c) (&sCf[s][0][0])[i] = Act<AT>::to_f32(rc[i]);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_ready[s]);
+            const int nxt = j + kStages - 1;  // goes into the stage that tile j - 1 occupied
+            if (nxt < ntiles) {
+                if (nxt >= kStages) ok = mbar_wait_bounded(&bar_empty[nxt % kStages], (uint32_t)(nxt / kStages - 1) & 1u);
+                if (!ok) break;
+                if (lane == 0) issue_tile(s_stage[nxt % kStages], &bar_raw[nxt % kStages], maps, ci.t0 + nxt * TT, d0, mask);
+                queued = nxt + 1;
+            }
+        }
+        if (!ok) {
+            if (lane == 0) flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
+            for (int j = landed; j < queued; ++j) mbar_wait_bounded(&bar_raw[j % kStages], (uint32_t)(j / kStages) & 1u);
+        }
+        return;
+    }
+
+    ChannelScan<AT, kPow, kOut, kFast> cs;
     if (live) {
         cs.init(p.L, d);
-        const AT* rows = nullptr;
-        if (ci.k == 0) {
-            if (ci.nck > 1 && !(p.L.flags & MDRAFT_PRECONV)) rows = static_cast<const AT*>(p.ws_conv) + (size_t)ci.seq * (kW - 1) * D;
-            else if (islot >= 0) rows = static_cast<const AT*>(p.pool.conv) + (size_t)islot * p.pool.conv_slot_stride;
+        const bool split = ci.nck > 1;
+        if (!preconv) {
+            const AT* rows = nullptr;
+            if (ci.k == 0) {
+                if (kOut && split) rows = static_cast<const AT*>(p.ws_conv) + (size_t)ci.seq * (kW - 1) * D;
+                else if (islot >= 0) rows = static_cast<const AT*>(p.pool.conv) + (size_t)islot * p.pool.conv_slot_stride;
+            }
+            load_window<AT>(cs.win, x, p.ldx, d, ci.t0, ci.k, rows, D);
         }
-        load_window<AT>(cs.win, x, p.ldx, d, ci.t0, ci.k, rows, D);
-        const float* hsrc = nullptr;
-        if (ci.k > 0) hsrc = p.ws_h + ((size_t)(cidx - 1) * D + d) * kN;
-        else if (islot >= 0) hsrc = p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)d * kN;
+        if (!kOut) {
+            if (ci.k == 0 && !preconv) {  // stash the starting window where the output pass will look for it
+                AT* stash = static_cast<AT*>(p.ws_conv) + (size_t)ci.seq * (kW - 1) * D;
 #pragma unroll
-        for (int q = 0; q < kN / 4; ++q) {
-            float4 v = hsrc ? *reinterpret_cast<const float4*>(hsrc + 4 * q) : make_float4(0.f, 0.f, 0.f, 0.f);
-            cs.h[4 * q] = v.x; cs.h[4 * q + 1] = v.y; cs.h[4 * q + 2] = v.z; cs.h[4 * q + 3] = v.w;
-        }
-    }
-    const bool conv_only = p.L.flags & MDRAFT_CONV_ONLY;
-    for (int t = ci.t0; t < ci.t1; t += kTT) {
-        int rows = min(kTT, ci.t1 - t);
-        __syncthreads();
-        if (!conv_only) stage_bc<AT>(sB, sC, B, C, p.ldb, p.ldc, t, rows, true);
-        __syncthreads();
-        if (live) {
-#pragma unroll 4
-            for (int r = 0; r < rows; ++r) {
-                float xv = Act<AT>::load(x + (size_t)(t + r) * p.ldx + d);
-                float zv = conv_only ? 0.0f : Act<AT>::load(z + (size_t)(t + r) * p.ldz + d);
-                float dtv = conv_only ? 0.0f : Act<AT>::load(dt + (size_t)(t + r) * p.lddt + d);
-                float o = cs.token(xv, zv, dtv, sB[r], sC[r]);
-                out[(size_t)(t + r) * p.ldo + d] = Act<AT>::from_f32(o);
+                for (int j = 0; j < kW - 1; ++j) stash[(size_t)j * D + d] = Act<AT>::from_f32(cs.win[j]);
+            }
+        } else if (!conv_only) {
+            // Incoming state: the slot itself for an unsplit sequence, else what the carry scan left.
+            const float4* src = nullptr;
+            size_t step = 1;
+            if (!split) {
+                if (islot >= 0) src = reinterpret_cast<const float4*>(p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)d * kN);
+            } else if (ci.k == 0) {
+                src = reinterpret_cast<const float4*>(p.ws_h0) + ((size_t)ci.seq * (kN / 4)) * D + d;
+                step = D;
+            } else {
+                src = reinterpret_cast<const float4*>(p.ws_q) + ((size_t)(cidx - 1) * (kN / 4)) * D + d;
+                step = D;
+            }
+            if (src) {
+#pragma unroll
+                for (int q = 0; q < kN / 4; ++q) {
+                    const float4 v = src[(size_t)q * step];
+                    cs.h[2 * q] = pk(v.x, v.y); cs.h[2 * q + 1] = pk(v.z, v.w);
+                }
             }
         }
     }
-    if (live && ci.k == ci.nck - 1 && fslot >= 0) {
+
+    // ---- channel warps
+    for (int j = 0; j < ntiles; ++j) {
+        const int s = j % kStages;
+        const int t = ci.t0 + j * TT;
+        const int rows = min(TT, ci.t1 - t);
+        const uint32_t parity = (uint32_t)(j / kStages) & 1u;
+        if (!mbar_wait_bounded(&bar_ready[s], parity) || !mbar_wait_bounded(&bar_raw[s], parity)) {
+            if (lane == 0) flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);  // the outputs of this chunk are invalid
+            return;
+        }
+        if (live) {
+            const unsigned char* st = s_stage[s];
+            const AT* sx = reinterpret_cast<const AT*>(st + kOffX) + tid;
+            const AT* sdt = reinterpret_cast<const AT*>(st + kOffDt) + tid;
+            const AT* sz = reinterpret_cast<const AT*>(st + kOffZ) + tid;
+            AT* orow = out + (size_t)t * p.ldo + d;
+#pragma unroll 4
+            for (int r = 0; r < rows; ++r) {
+                const float xv = Act<AT>::to_f32(sx[r * kCB]);
+                const float dtv = conv_only ? 0.0f : Act<AT>::to_f32(sdt[r * kCB]);
+                const float zv = want_c ? Act<AT>::to_f32(sz[r * kCB]) : 0.0f;
+                const float o = cs.token(xv, zv, dtv, sBf[s][r], sCf[s][r]);
+                if (kOut) orow[(size_t)r * p.ldo] = Act<AT>::from_f32(o);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_empty[s]);
+    }
+
+    if (!live) return;
+    if (!kOut) {
+        if (compute) {
+            float4* dst = reinterpret_cast<float4*>(p.ws_q) + ((size_t)cidx * (kN / 4)) * D + d;
+#pragma unroll
+            for (int q = 0; q < kN / 4; ++q) {
+                float a, b, c, e;
+                unpk(cs.h[2 * q], a, b);
+                unpk(cs.h[2 * q + 1], c, e);
+                dst[(size_t)q * D] = make_float4(a, b, c, e);
+            }
+            p.ws_sd[(size_t)cidx * D + d] = cs.sum_delta;
+        }
+        return;
+    }
+    if (ci.k == ci.nck - 1 && fslot >= 0) {
         if (!conv_only) {
             float4* dst = reinterpret_cast<float4*>(p.pool.ssm + (size_t)fslot * p.pool.ssm_slot_stride + (size_t)d * kN);
 #pragma unroll
-            for (int q = 0; q < kN / 4; ++q) dst[q] = make_float4(cs.h[4 * q], cs.h[4 * q + 1], cs.h[4 * q + 2], cs.h[4 * q + 3]);
+            for (int q = 0; q < kN / 4; ++q) {
+                float a, b, c, e;
+                unpk(cs.h[2 * q], a, b);
+                unpk(cs.h[2 * q + 1], c, e);
+                dst[q] = make_float4(a, b, c, e);
+            }
         }
-        if (!(p.L.flags & MDRAFT_PRECONV)) {
+        if (!preconv) {
             AT* dc = static_cast<AT*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride;
 #pragma unroll
             for (int j = 0; j < kW - 1; ++j) dc[(size_t)j * D + d] = Act<AT>::from_f32(cs.win[j]);
@@ -422,33 +540,102 @@ __global__ void __launch_bounds__(kPrefillThreads) chunk_scan_kernel(PrefillArgs
     }
 }
 
-template <typename AT, bool kPow>
-cudaError_t launch_typed(const PrefillArgs& p, bool chunked, cudaStream_t st) {
+// ---------------------------------------------------------------------------------------------------
+// Carry scan.  Block = 8 warps; a warp's lanes are 32 consecutive floats of one state quad (8 channels x 4
+// entries), so every load and store of a warp is one 128-byte line.  Per round, warp g takes kCarryPer
+// consecutive chunks: it loads their summaries at once, folds them into one (P, q) pair, publishes the pair,
+// folds the pairs of the warps before it into its starting state, and then replays its own chunks to write the
+// state after each.  Rounds carry the running state forward for sequences of more than 64 chunks.
+constexpr int kCarryGroups = 8, kCarryPer = 8;
+
+__global__ void __launch_bounds__(kCarryGroups * 32) carry_kernel(PrefillArgs p) {
+    __shared__ float sP[kCarryGroups][32];
+    __shared__ float sQ[kCarryGroups][32];
     const int D = p.L.d_inner;
-    dim3 grid((D + kPrefillThreads - 1) / kPrefillThreads, p.n_chunks_bound);
-    const bool recur = !(p.L.flags & MDRAFT_CONV_ONLY);
-    if (chunked) {
-        chunk_state_kernel<AT, kPow><<<grid, kPrefillThreads, 0, st>>>(p);
-        if (p.ev_state) cudaEventRecord(p.ev_state, st);
-        if (recur) {
-            dim3 g2((D * kN + 31) / 32, p.n_seq);
-            carry_scan_kernel<<<g2, 1024, 0, st>>>(p);
+    const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
+    const int quad = blockIdx.y, s = blockIdx.z;
+    const int d = blockIdx.x * 8 + (lane >> 2);  // d_inner is a multiple of 8
+    const int n = quad * 4 + (lane & 3);
+    int first, nck;
+    seq_chunks(p.cu, p.n_seq, p.T, p.chunk_len, s, first, nck);
+    if (nck <= 1) return;
+    const int islot = load_slot(p.init_slot, s), fslot = load_slot(p.final_slot, s);
+    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;  // the output pass reports it
+
+    const float a2 = __ldg(p.L.A + (size_t)d * kN + n) * kLog2e;
+    float carry = islot >= 0 ? p.pool.ssm[(size_t)islot * p.pool.ssm_slot_stride + (size_t)d * kN + n] : 0.0f;
+    const size_t col = (size_t)quad * D * 4 + (size_t)d * 4 + (lane & 3);  // offset inside one chunk's [N/4][D][4] block
+    const size_t per_chunk = (size_t)D * kN;
+    if (g == 0) p.ws_h0[(size_t)s * per_chunk + col] = carry;
+
+    const int nsum = nck - 1;  // summaries of chunks 0 .. nck-2
+    for (int base = 0; base < nsum; base += kCarryGroups * kCarryPer) {
+        const int c0 = base + g * kCarryPer;
+        float q[kCarryPer], a[kCarryPer];
+#pragma unroll
+        for (int i = 0; i < kCarryPer; ++i) {
+            const int c = c0 + i;
+            q[i] = 0.0f; a[i] = 0.0f;
+            if (c < nsum) {
+                q[i] = p.ws_q[(size_t)(first + c) * per_chunk + col];
+                a[i] = p.ws_sd[(size_t)(first + c) * D + d];
+            }
         }
-        if (p.ev_carry) cudaEventRecord(p.ev_carry, st);
-    } else {
-        if (p.ev_state) cudaEventRecord(p.ev_state, st);
-        if (p.ev_carry) cudaEventRecord(p.ev_carry, st);
+        float Pg = 1.0f, qg = 0.0f;
+#pragma unroll
+        for (int i = 0; i < kCarryPer; ++i) {
+            a[i] = ex2(a2 * a[i]);  // sum of Delta -> decay of the whole chunk (1 for the padding past nsum)
+            qg = fmaf(a[i], qg, q[i]);
+            Pg *= a[i];
+        }
+        sP[g][lane] = Pg;
+        sQ[g][lane] = qg;
+        __syncthreads();
+        float h = carry;
+        for (int gg = 0; gg < g; ++gg) h = fmaf(sP[gg][lane], h, sQ[gg][lane]);
+        float after = h;  // running state after the whole round, the same in every warp
+        for (int gg = g; gg < kCarryGroups; ++gg) after = fmaf(sP[gg][lane], after, sQ[gg][lane]);
+#pragma unroll
+        for (int i = 0; i < kCarryPer; ++i) {
+            const int c = c0 + i;
+            if (c < nsum) {
+                h = fmaf(a[i], h, q[i]);
+                p.ws_q[(size_t)(first + c) * per_chunk + col] = h;
+            }
+        }
+        carry = after;
+        __syncthreads();
     }
-    chunk_scan_kernel<AT, kPow><<<grid, kPrefillThreads, 0, st>>>(p);
+}
+
+template <typename AT, bool kPow, bool kFast>
+cudaError_t launch_typed(const PrefillArgs& p, const PrefillMaps& maps, bool chunked, cudaStream_t st) {
+    const int D = p.L.d_inner;
+    dim3 grid((D + kCB - 1) / kCB, p.n_chunks_bound);
+    const bool recur = !(p.L.flags & MDRAFT_CONV_ONLY);
+    if (chunked) chunk_kernel<AT, kPow, false, kFast><<<grid, kBlockThreads, 0, st>>>(p, maps);
+    if (p.ev_state) cudaEventRecord(p.ev_state, st);
+    if (chunked && recur) {
+        dim3 g2(D / 8, kN / 4, p.n_seq);
+        carry_kernel<<<g2, kCarryGroups * 32, 0, st>>>(p);
+    }
+    if (p.ev_carry) cudaEventRecord(p.ev_carry, st);
+    chunk_kernel<AT, kPow, true, kFast><<<grid, kBlockThreads, 0, st>>>(p, maps);
     return cudaGetLastError();
+}
+
+template <typename AT>
+cudaError_t launch_act(const PrefillArgs& p, const PrefillMaps& maps, bool chunked, cudaStream_t st) {
+    const bool pow = p.L.flags & MDRAFT_A_POWERS;
+    const bool fast = (p.L.flags & ~(uint32_t)MDRAFT_A_POWERS) == (uint32_t)MDRAFT_DT_SOFTPLUS;
+    if (fast) return pow ? launch_typed<AT, true, true>(p, maps, chunked, st) : launch_typed<AT, false, true>(p, maps, chunked, st);
+    return pow ? launch_typed<AT, true, false>(p, maps, chunked, st) : launch_typed<AT, false, false>(p, maps, chunked, st);
 }
 
 }  // namespace
 
-cudaError_t launch_prefill(const PrefillArgs& p, int act, bool chunked, cudaStream_t st) {
-    const bool pow = p.L.flags & MDRAFT_A_POWERS;
-    if (act == MDRAFT_F32) return pow ? launch_typed<float, true>(p, chunked, st) : launch_typed<float, false>(p, chunked, st);
-    return pow ? launch_typed<__nv_bfloat16, true>(p, chunked, st) : launch_typed<__nv_bfloat16, false>(p, chunked, st);
+cudaError_t launch_prefill(const PrefillArgs& p, const PrefillMaps& maps, int act, bool chunked, cudaStream_t st) {
+    return act == MDRAFT_F32 ? launch_act<float>(p, maps, chunked, st) : launch_act<__nv_bfloat16>(p, maps, chunked, st);
 }
 
 }  // namespace mdraft

@@ -1,6 +1,8 @@
 // Launch interface of the prefill kernels (internal to the library).
 #pragma once
 
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace mdraft {
@@ -15,13 +17,23 @@ struct PrefillArgs {
     int64_t ldx, ldz, lddt, ldb, ldc, ldo;
     int T, n_seq, chunk_len, n_chunks_bound;
     const int32_t *cu, *init_slot, *final_slot;
-    float* ws_h;    // [n_chunks_bound][D][N] chunk summaries, then incoming states
-    float* ws_sd;   // [n_chunks_bound][D]    sum of Delta per chunk
-    void* ws_conv;  // [n_seq][W-1][D]        starting conv windows (activation type)
+    float* ws_q;    // [n_chunks_bound][N/4][D][4] zero-state result of each chunk; after the carry scan, entry c holds
+                    //                             the state after chunk c = the incoming state of chunk c + 1
+    float* ws_sd;   // [n_chunks_bound][D]         sum of Delta per chunk
+    float* ws_h0;   // [n_seq][N/4][D][4]          starting state of each split sequence
+    void* ws_conv;  // [n_seq][W-1][D]             starting conv window of each split sequence (activation type)
     int32_t* dev_status;
     cudaEvent_t ev_state, ev_carry;  // optional profiling events (host side only)
 };
 
-cudaError_t launch_prefill(const PrefillArgs& p, int act, bool chunked, cudaStream_t st);
+constexpr int kPrefillTileRowBytes = 32;  // a staged tile holds 32 / sizeof(activation) tokens: 16 (bf16) or 8 (fp32)
+
+// TMA descriptors of the five activation matrices of one call: boxes of kPrefillThreads channels (x, dt, z) or
+// 16 values (B, C) by one tile of tokens.  Built on the host for every call (they hold the base addresses).
+struct PrefillMaps {
+    CUtensorMap x, dt, z, B, C;
+};
+
+cudaError_t launch_prefill(const PrefillArgs& p, const PrefillMaps& maps, int act, bool chunked, cudaStream_t st);
 
 }  // namespace mdraft
