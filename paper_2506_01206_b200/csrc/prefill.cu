@@ -101,6 +101,14 @@ __device__ __forceinline__ void tma_box(void* dst, const CUtensorMap* map, int c
                  : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// The three kernels of a call (and the first kernel of the next call on the stream) are launched with programmatic
+// stream serialisation: a kernel may start while its predecessor is still running, and must pass grid_wait() before
+// it touches anything the predecessor (or a kernel before that) writes, or overwrites anything it reads.  Every block
+// passes grid_wait() on every path, so that a kernel's completion implies that of all its predecessors.
+__device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- chunk bookkeeping
 struct ChunkInfo {
     int seq;     // sequence index, -1 if this chunk id is past the last chunk
@@ -330,6 +338,11 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
     const uint32_t flags = kFast ? (uint32_t)MDRAFT_DT_SOFTPLUS : p.L.flags;
     const bool conv_only = flags & MDRAFT_CONV_ONLY, preconv = flags & MDRAFT_PRECONV;
 
+    // Layer constants first: they depend on nothing but the channel and are never written by a kernel of this
+    // library, so they may be read before the predecessor on the stream has finished.
+    ChannelScan<AT, kPow, kOut, kFast> cs;
+    if (live) cs.init(p.L, d);
+
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < kStages; ++s) {
@@ -340,10 +353,20 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    if (!kOut) {
+        // Summary pass: the inputs may be the work of the kernel before this call, so nothing else is read before
+        // that kernel is known to be complete; only then may the kernels after this one start.
+        grid_wait();
+        grid_release_dependents();
+    } else {
+        grid_release_dependents();
+        if (!p.pdl_inputs_ready) grid_wait();  // unsplit call: no summary pass has waited for the inputs yet
+    }
 
     if (kOut) {
         // Sequences without tokens have no chunk: their final state is their starting state.
         if (cidx == 0 && p.final_slot) {
+            grid_wait();  // the state pool may be the work of the kernels before
             for (int s = 0; s < p.n_seq; ++s) {
                 int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
                 bool bad = (lo < 0) || (hi < lo) || (hi > p.T);
@@ -373,19 +396,12 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
     }
 
     const ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, p.chunk_len, cidx);
-    if (ci.seq < 0) return;
+    if (ci.seq < 0) { if (kOut) grid_wait(); return; }
     if (!kOut) {
         // No summary is needed for an unsplit sequence or for a sequence's last chunk; in conv-only mode the only
         // job left is the first chunk's stash of the starting window.
         if (ci.nck == 1 || ci.k == ci.nck - 1) return;
         if ((flags & MDRAFT_CONV_ONLY) && ci.k > 0) return;
-    }
-
-    const int islot = load_slot(p.init_slot, ci.seq);
-    const int fslot = load_slot(p.final_slot, ci.seq);
-    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) {  // whole sequence becomes a no-op
-        if (kOut && tid == 0 && blockIdx.x == 0 && ci.k == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
-        return;
     }
 
     const AT* x = static_cast<const AT*>(p.x);
@@ -398,11 +414,22 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
     if (!conv_only) mask = kOut ? 15u : 5u;  // summary pass: x, dt, B
 
     const bool want_c = kOut && !conv_only;
+    const int pre = min(kStages - 1, ntiles);
+    if (copy_warp && lane == 0)  // the first tiles go out before anything else is looked up
+        for (int j = 0; j < pre; ++j) issue_tile(s_stage[j], &bar_raw[j], maps, ci.t0 + j * TT, d0, mask);
+
+    const int islot = load_slot(p.init_slot, ci.seq);
+    const int fslot = load_slot(p.final_slot, ci.seq);
+    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) {  // whole sequence becomes a no-op
+        if (kOut && tid == 0 && blockIdx.x == 0 && ci.k == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+        if (copy_warp)  // the tiles already queued still land in this block's shared memory: see them in first
+            for (int j = 0; j < pre; ++j) mbar_wait_bounded(&bar_raw[j], 0u);
+        if (kOut) grid_wait();
+        return;
+    }
+
     if (copy_warp) {
         // ---- copy warp: keep two tiles in flight, widen B / C of each landed tile, hand it over.
-        const int pre = min(kStages - 1, ntiles);
-        if (lane == 0)
-            for (int j = 0; j < pre; ++j) issue_tile(s_stage[j], &bar_raw[j], maps, ci.t0 + j * TT, d0, mask);
         int landed = 0, queued = pre;  // tiles [landed, queued) are in flight
         bool ok = true;
         for (int j = 0; j < ntiles && ok; ++j) {
@@ -433,12 +460,13 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
             if (lane == 0) flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
             for (int j = landed; j < queued; ++j) mbar_wait_bounded(&bar_raw[j % kStages], (uint32_t)(j / kStages) & 1u);
         }
+        if (kOut) grid_wait();
         return;
     }
 
-    ChannelScan<AT, kPow, kOut, kFast> cs;
+    // Output pass: everything read from here on (workspace, state pool) may be the work of the kernels just before.
+    if (kOut) grid_wait();
     if (live) {
-        cs.init(p.L, d);
         const bool split = ci.nck > 1;
         if (!preconv) {
             const AT* rows = nullptr;
@@ -541,66 +569,77 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Carry scan.  Block = 8 warps; a warp's lanes are 32 consecutive floats of one state quad (8 channels x 4
-// entries), so every load and store of a warp is one 128-byte line.  Per round, warp g takes kCarryPer
-// consecutive chunks: it loads their summaries at once, folds them into one (P, q) pair, publishes the pair,
-// folds the pairs of the warps before it into its starting state, and then replays its own chunks to write the
-// state after each.  Rounds carry the running state forward for sequences of more than 64 chunks.
-constexpr int kCarryGroups = 8, kCarryPer = 8;
+// Carry scan.  Block = 8 warps; a thread owns one state quad (4 entries of one channel), a warp's lanes are 32
+// consecutive channels of that quad, so every load and store of a warp is 512 contiguous bytes.  Per round,
+// warp g takes kCarryPer consecutive chunks: it loads their summaries at once, folds them into one (P, q) pair,
+// publishes the pair, folds the pairs of the warps before it into its starting state, and then replays its own
+// chunks to write the state after each.  Rounds carry the running state forward past 48 chunks.
+constexpr int kCarryGroups = 8, kCarryPer = 6;
 
-__global__ void __launch_bounds__(kCarryGroups * 32) carry_kernel(PrefillArgs p) {
-    __shared__ float sP[kCarryGroups][32];
-    __shared__ float sQ[kCarryGroups][32];
+__device__ __forceinline__ float4 fold4(const float4& a, const float4& h, const float4& q) {
+    return make_float4(fmaf(a.x, h.x, q.x), fmaf(a.y, h.y, q.y), fmaf(a.z, h.z, q.z), fmaf(a.w, h.w, q.w));
+}
+
+__global__ void __launch_bounds__(kCarryGroups * 32) carry_kernel(const PrefillArgs p) {
+    __shared__ float4 sP[kCarryGroups][32];
+    __shared__ float4 sQ[kCarryGroups][32];
     const int D = p.L.d_inner;
     const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
     const int quad = blockIdx.y, s = blockIdx.z;
-    const int d = blockIdx.x * 8 + (lane >> 2);  // d_inner is a multiple of 8
-    const int n = quad * 4 + (lane & 3);
+    const int d = blockIdx.x * 32 + lane;
+    const bool live = d < D;
+    const int dd = live ? d : 0;  // dead lanes shadow channel 0 and write nothing
+    float4 a2 = __ldg(reinterpret_cast<const float4*>(p.L.A + (size_t)dd * kN) + quad);
+    a2.x *= kLog2e; a2.y *= kLog2e; a2.z *= kLog2e; a2.w *= kLog2e;
+    grid_release_dependents();
+    grid_wait();  // the summaries are the work of the kernel just before
+
     int first, nck;
     seq_chunks(p.cu, p.n_seq, p.T, p.chunk_len, s, first, nck);
     if (nck <= 1) return;
     const int islot = load_slot(p.init_slot, s), fslot = load_slot(p.final_slot, s);
     if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;  // the output pass reports it
 
-    const float a2 = __ldg(p.L.A + (size_t)d * kN + n) * kLog2e;
-    float carry = islot >= 0 ? p.pool.ssm[(size_t)islot * p.pool.ssm_slot_stride + (size_t)d * kN + n] : 0.0f;
-    const size_t col = (size_t)quad * D * 4 + (size_t)d * 4 + (lane & 3);  // offset inside one chunk's [N/4][D][4] block
-    const size_t per_chunk = (size_t)D * kN;
-    if (g == 0) p.ws_h0[(size_t)s * per_chunk + col] = carry;
+    float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (islot >= 0) carry = *(reinterpret_cast<const float4*>(p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)dd * kN) + quad);
+    const size_t per_chunk = (size_t)D * (kN / 4);  // float4s in one chunk's [N/4][D] block
+    const size_t col = (size_t)quad * D + dd;        // this thread's float4 inside such a block
+    float4* wsq = reinterpret_cast<float4*>(p.ws_q);
+    if (g == 0 && live) reinterpret_cast<float4*>(p.ws_h0)[(size_t)s * per_chunk + col] = carry;
 
     const int nsum = nck - 1;  // summaries of chunks 0 .. nck-2
     for (int base = 0; base < nsum; base += kCarryGroups * kCarryPer) {
         const int c0 = base + g * kCarryPer;
-        float q[kCarryPer], a[kCarryPer];
+        const int cnt = min(kCarryPer, nsum - c0);  // may be <= 0
+        float4 q[kCarryPer], a[kCarryPer];
+        const float4* qp = wsq + (size_t)(first + c0) * per_chunk + col;
+        const float* sp = p.ws_sd + (size_t)(first + c0) * D + dd;
 #pragma unroll
         for (int i = 0; i < kCarryPer; ++i) {
-            const int c = c0 + i;
-            q[i] = 0.0f; a[i] = 0.0f;
-            if (c < nsum) {
-                q[i] = p.ws_q[(size_t)(first + c) * per_chunk + col];
-                a[i] = p.ws_sd[(size_t)(first + c) * D + d];
-            }
+            q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            float sd = 0.0f;  // padding past nsum: decay 1, nothing added
+            if (i < cnt) { q[i] = qp[(size_t)i * per_chunk]; sd = sp[(size_t)i * D]; }
+            a[i] = make_float4(ex2(a2.x * sd), ex2(a2.y * sd), ex2(a2.z * sd), ex2(a2.w * sd));  // decay of the whole chunk
         }
-        float Pg = 1.0f, qg = 0.0f;
+        float4 Pg = make_float4(1.f, 1.f, 1.f, 1.f), qg = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int i = 0; i < kCarryPer; ++i) {
-            a[i] = ex2(a2 * a[i]);  // sum of Delta -> decay of the whole chunk (1 for the padding past nsum)
-            qg = fmaf(a[i], qg, q[i]);
-            Pg *= a[i];
+            qg = fold4(a[i], qg, q[i]);
+            Pg.x *= a[i].x; Pg.y *= a[i].y; Pg.z *= a[i].z; Pg.w *= a[i].w;
         }
         sP[g][lane] = Pg;
         sQ[g][lane] = qg;
         __syncthreads();
-        float h = carry;
-        for (int gg = 0; gg < g; ++gg) h = fmaf(sP[gg][lane], h, sQ[gg][lane]);
-        float after = h;  // running state after the whole round, the same in every warp
-        for (int gg = g; gg < kCarryGroups; ++gg) after = fmaf(sP[gg][lane], after, sQ[gg][lane]);
+        float4 h = carry;
+        for (int gg = 0; gg < g; ++gg) h = fold4(sP[gg][lane], h, sQ[gg][lane]);
+        float4 after = h;  // running state after the whole round, the same in every warp
+        for (int gg = g; gg < kCarryGroups; ++gg) after = fold4(sP[gg][lane], after, sQ[gg][lane]);
+        float4* op = wsq + (size_t)(first + c0) * per_chunk + col;
 #pragma unroll
         for (int i = 0; i < kCarryPer; ++i) {
-            const int c = c0 + i;
-            if (c < nsum) {
-                h = fmaf(a[i], h, q[i]);
-                p.ws_q[(size_t)(first + c) * per_chunk + col] = h;
+            if (i < cnt) {
+                h = fold4(a[i], h, q[i]);
+                if (live) op[(size_t)i * per_chunk] = h;
             }
         }
         carry = after;
@@ -608,19 +647,40 @@ __global__ void __launch_bounds__(kCarryGroups * 32) carry_kernel(PrefillArgs p)
     }
 }
 
+// Launch with programmatic stream serialisation: the kernel may begin before the one ahead of it has finished.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <typename AT, bool kPow, bool kFast>
-cudaError_t launch_typed(const PrefillArgs& p, const PrefillMaps& maps, bool chunked, cudaStream_t st) {
+cudaError_t launch_typed(PrefillArgs p, const PrefillMaps& maps, bool chunked, cudaStream_t st) {
     const int D = p.L.d_inner;
     dim3 grid((D + kCB - 1) / kCB, p.n_chunks_bound);
     const bool recur = !(p.L.flags & MDRAFT_CONV_ONLY);
-    if (chunked) chunk_kernel<AT, kPow, false, kFast><<<grid, kBlockThreads, 0, st>>>(p, maps);
+    p.pdl_inputs_ready = chunked ? 1 : 0;  // the summary pass waits for the producer of the inputs on behalf of all three
+    cudaError_t e = cudaSuccess;
+    if (chunked) e = launch_pdl(chunk_kernel<AT, kPow, false, kFast>, grid, kBlockThreads, st, p, maps);
+    if (e != cudaSuccess) return e;
     if (p.ev_state) cudaEventRecord(p.ev_state, st);
     if (chunked && recur) {
-        dim3 g2(D / 8, kN / 4, p.n_seq);
-        carry_kernel<<<g2, kCarryGroups * 32, 0, st>>>(p);
+        dim3 g2((D + 31) / 32, kN / 4, p.n_seq);
+        e = launch_pdl(carry_kernel, g2, kCarryGroups * 32, st, p);
+        if (e != cudaSuccess) return e;
     }
     if (p.ev_carry) cudaEventRecord(p.ev_carry, st);
-    chunk_kernel<AT, kPow, true, kFast><<<grid, kBlockThreads, 0, st>>>(p, maps);
+    e = launch_pdl(chunk_kernel<AT, kPow, true, kFast>, grid, kBlockThreads, st, p, maps);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 

@@ -23,6 +23,7 @@ struct PrefillArgs {
     float* ws_h0;   // [n_seq][N/4][D][4]          starting state of each split sequence
     void* ws_conv;  // [n_seq][W-1][D]             starting conv window of each split sequence (activation type)
     int32_t* dev_status;
+    int pdl_inputs_ready;  // set by the launcher: 1 if an earlier kernel of this call has already waited for the inputs
     cudaEvent_t ev_state, ev_carry;  // optional profiling events (host side only)
 };
 
