@@ -5,7 +5,7 @@
 
 namespace mdraft {
 
-constexpr int kTreeThreads = 128;  // 32 channels x 4 lanes per channel
+constexpr int kTreeThreads = 128;  // channels per block, one thread each
 
 struct TreeArgs {
     LayerDev L;
