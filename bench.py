@@ -217,36 +217,26 @@ class BatchedTree:
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
-
     import paper_2506_01206_b200 as md
+    from paper_2506_01206_b200 import replicas
     from paper_2506_01206_b200.device_inputs import i32, to_device, torch_act, upload_layer
     from paper_2506_01206_b200.stack import DrafterStack
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = replicas.env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init("nccl", dev)
     md.load_library()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(world)
 
     def max_over_ranks(v: float) -> float:
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(v, world, dev)
 
-    w = Workload(seed=rank, n_layers=24)
+    w = Workload(seed=replicas.replica_seed(0, rank), n_layers=24)
     tdt = torch_act(w.cfg.act)
     T, M, D, NL = w.T, w.M, w.cfg.d_inner, w.n_layers
 
@@ -402,7 +392,7 @@ def run_ours(args):
 
     units_step = NL * T * D                      # prefill token*channels per step per GPU
     node_updates = NL * M
-    value = world * units_step / (ms_step * 1e-3)
+    value = replicas.whole_job_throughput(units_step, ms_step, world)
     peak, peak_src = load_peaks()
     pre_launches = stack.prefill_launches_per_layer(T, 1, T)
     launches = NL * pre_launches + NL * (len(levels) - 1) + 1
@@ -489,8 +479,7 @@ def run_ours(args):
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish(world)
 
 
 def main():
