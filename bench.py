@@ -185,6 +185,10 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------- GPU leg
 ALU_LANE_OPS_PER_UNIT = 82      # fp32 lane-operations per token*channel of a single-pass prefill (derivation in the design doc)
 FP32_LANES_PER_SM, SM_COUNT = 128, 148
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/ (set to None
+# whenever the kernel changes after the counters were taken)
+NCU_TRAFFIC_OUTPUT_PASS = 24.01e6   # chunk_kernel<bf16, structured A, output pass>, 2048 x 1536
+NCU_TRAFFIC_TREE_WIDEST = 31.53e6   # tree_step_kernel<bf16>, 442-node level of the 32 x 32-node round
 
 
 class BatchedTree:
@@ -407,7 +411,7 @@ def run_ours(args):
     kname = "chunk_kernel<bf16, %s, output pass>" % ("structured A" if is_pow else "general A")
     roofline = {
         "bound": "hbm", "kernel": kname, "achieved": pb / scan_s / 1e9, "peak": peak, "unit": "GB/s",
-        "frac": pb / scan_s / 1e9 / peak, "traffic": None, "peak_source": peak_src,
+        "frac": pb / scan_s / 1e9 / peak, "traffic": NCU_TRAFFIC_OUTPUT_PASS, "peak_source": peak_src,
         "frac_of_nominal_8000": pb / scan_s / 1e9 / 8000.0, "algorithmic_bytes_per_launch": pb, "launch_us": split[2],
         "timed": "CUDA events recorded by the library between the kernels of each layer's call, host queued ahead of the GPU; median of 72 calls",
         "alu": {"achieved": ALU_LANE_OPS_PER_UNIT * T * D / scan_s / 1e12, "peak": alu_peak / 1e12, "unit": "T fp32 lane-op/s",
@@ -423,7 +427,7 @@ def run_ours(args):
     roofline_tree = {
         "bound": "hbm", "kernel": "tree_step_kernel<bf16>", "workload": "32 sequences x 32-node trees, widest level (%d nodes), 24 layers" % (hi - lo),
         "achieved": NL * bt_wide_bytes / (ms_bt_widest * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
-        "frac": NL * bt_wide_bytes / (ms_bt_widest * 1e-3) / 1e9 / peak, "traffic": None,
+        "frac": NL * bt_wide_bytes / (ms_bt_widest * 1e-3) / 1e9 / peak, "traffic": NCU_TRAFFIC_TREE_WIDEST,
         "algorithmic_bytes_per_launch": bt_wide_bytes, "launch_us": 1e3 * ms_bt_widest / NL,
         "timed": "CUDA-graph replay of 24 launches (one per layer, distinct 110 MB pools), time / 24",
         "whole_round": {"ms": ms_bt_round, "levels": [b - a for a, b in zip(bt.levels[:-1], bt.levels[1:])],
