@@ -265,7 +265,7 @@ def run_ours(args):
     stack = make_stack(md.MDRAFT_A_POWERS if is_pow else 0, w.params)
     stack_general = make_stack(0, w.params)
 
-    cu = i32([0, T], dev)
+    cu = None  # one sequence of all T rows: the library needs no offsets for that
     slot0 = i32([0], dev)
     parent_slot = i32(np.where(w.tree.parents < 0, 0, w.tree.parents + 1), dev)
     node_slot = i32(np.arange(M) + 1, dev)

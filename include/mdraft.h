@@ -130,7 +130,9 @@ typedef struct {
  *   x, z, dt : (T, D) activations, strides ldx, ldz, lddt           [read]
  *   B, C     : (T, N) activations, strides ldb, ldc                 [read]
  *   out      : (T, D) activations, stride ldo                       [written]
- *   cu_seqlens : n_seq+1 int32, tokens of sequence s are rows cu_seqlens[s] .. cu_seqlens[s+1]-1
+ *   cu_seqlens : n_seq+1 int32, tokens of sequence s are rows cu_seqlens[s] .. cu_seqlens[s+1]-1.  May be NULL
+ *                when n_seq == 1: the one sequence is then rows 0 .. total_tokens-1, and no kernel has to
+ *                fetch offsets from memory before it can start
  *   init_slot  : n_seq int32 or NULL; slot holding each sequence's starting state, -1 / NULL = zero state
  *   final_slot : n_seq int32 or NULL; slot that receives the state after the last token, -1 / NULL = discard.
  *                init_slot[s] == final_slot[s] is allowed (encode a context in pieces).

@@ -201,7 +201,7 @@ def mdraft_prefill_workspace_bytes(layer: Layer, total_tokens: int, n_seq: int, 
 
 
 def mdraft_conv_scan_prefill(layer: Layer, cache: Optional[StateCache], layer_index: int,
-                             x, z, dt, B, Cm, out, cu_seqlens: torch.Tensor, max_seqlen: int,
+                             x, z, dt, B, Cm, out, cu_seqlens: Optional[torch.Tensor], max_seqlen: int,
                              init_slot: Optional[torch.Tensor] = None, final_slot: Optional[torch.Tensor] = None,
                              workspace: Optional[torch.Tensor] = None, chunk_len: int = 0,
                              dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None,
@@ -212,8 +212,8 @@ def mdraft_conv_scan_prefill(layer: Layer, cache: Optional[StateCache], layer_in
     px, ldx = _mat(x, "x"); pz, ldz = _mat(z, "z"); pdt, lddt = _mat(dt, "dt")
     pB, ldb = _mat(B, "B"); pC, ldc = _mat(Cm, "C"); po, ldo = _mat(out, "out")
     T = int(x.shape[0])
-    n_seq = int(cu_seqlens.numel()) - 1
-    if cu_seqlens.dtype != torch.int32:
+    n_seq = 1 if cu_seqlens is None else int(cu_seqlens.numel()) - 1   # None: a single sequence of all T rows
+    if cu_seqlens is not None and cu_seqlens.dtype != torch.int32:
         raise TypeError("cu_seqlens must be int32")
     for t, nm in ((init_slot, "init_slot"), (final_slot, "final_slot")):
         if t is not None and (t.dtype != torch.int32 or t.numel() != n_seq):
@@ -231,7 +231,7 @@ NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 def mdraft_conv_scan_prefill_noalloc(layer: Layer, cache: Optional[StateCache], layer_index: int,
-                                     x, z, dt, B, Cm, out, cu_seqlens: torch.Tensor, max_seqlen: int,
+                                     x, z, dt, B, Cm, out, cu_seqlens: Optional[torch.Tensor], max_seqlen: int,
                                      init_slot: Optional[torch.Tensor] = None, final_slot: Optional[torch.Tensor] = None,
                                      chunk_len: int = 0, dev_status: Optional[torch.Tensor] = None, stream=None,
                                      flags: Optional[int] = None) -> None:
@@ -244,8 +244,8 @@ def mdraft_conv_scan_prefill_noalloc(layer: Layer, cache: Optional[StateCache], 
     px, ldx = _mat(x, "x"); pz, ldz = _mat(z, "z"); pdt, lddt = _mat(dt, "dt")
     pB, ldb = _mat(B, "B"); pC, ldc = _mat(Cm, "C"); po, ldo = _mat(out, "out")
     T = int(x.shape[0])
-    n_seq = int(cu_seqlens.numel()) - 1
-    if cu_seqlens.dtype != torch.int32:
+    n_seq = 1 if cu_seqlens is None else int(cu_seqlens.numel()) - 1   # None: a single sequence of all T rows
+    if cu_seqlens is not None and cu_seqlens.dtype != torch.int32:
         raise TypeError("cu_seqlens must be int32")
     for t, nm in ((init_slot, "init_slot"), (final_slot, "final_slot")):
         if t is not None and (t.dtype != torch.int32 or t.numel() != n_seq):

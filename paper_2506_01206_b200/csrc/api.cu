@@ -193,11 +193,8 @@ int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cach
         rc = check_cache(cache, layer->d_inner, layer->act, layer_index);
         if (rc) return rc;
     }
-    if (n_seq == 0 || total_tokens == 0) {
-        if (n_seq > 0 && !cu_seqlens) return MDRAFT_ERR_INVALID_ARG;
-        if (n_seq == 0) return MDRAFT_OK;
-    }
-    if (!cu_seqlens) return MDRAFT_ERR_INVALID_ARG;
+    if (n_seq == 0) return MDRAFT_OK;
+    if (!cu_seqlens && n_seq != 1) return MDRAFT_ERR_INVALID_ARG;  // offsets may be omitted for a single sequence only
     const bool conv_only = layer->flags & MDRAFT_CONV_ONLY;
     const int D = layer->d_inner, act = layer->act;
     const bool have_rows = total_tokens > 0;

@@ -122,6 +122,10 @@ struct ChunkInfo {
 // gets none.  Global chunk ids number the chunks of sequence 0, then 1, ...  Called by whole warps.
 __device__ __forceinline__ void seq_span(const int32_t* cu, int n_seq, int T, int s, int& a, int& len, bool& bad) {
     a = 0; len = 0; bad = false;
+    if (!cu) {  // no offsets given: one sequence that is all T rows (nothing to look up in memory)
+        if (s == 0) len = T;
+        return;
+    }
     if (s < n_seq) {
         int lo = __ldg(cu + s), hi = __ldg(cu + s + 1);
         bad = (lo < 0) || (hi < lo) || (hi > T);
@@ -368,7 +372,7 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
         if (cidx == 0 && p.final_slot) {
             grid_wait();  // the state pool may be the work of the kernels before
             for (int s = 0; s < p.n_seq; ++s) {
-                int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
+                int lo = p.cu ? __ldg(p.cu + s) : 0, hi = p.cu ? __ldg(p.cu + s + 1) : p.T;
                 bool bad = (lo < 0) || (hi < lo) || (hi > p.T);
                 if (bad && blockIdx.x == 0 && tid == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);
                 if (bad || hi != lo) continue;
@@ -387,7 +391,7 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
                     for (int j = 0; j < kW - 1; ++j) dc[(size_t)j * D + d] = sc ? sc[(size_t)j * D + d] : Act<AT>::from_f32(0.0f);
                 }
             }
-        } else if (cidx == 0 && blockIdx.x == 0 && tid < 32) {
+        } else if (cidx == 0 && blockIdx.x == 0 && tid < 32 && p.cu) {
             for (int s = tid; s < p.n_seq; s += 32) {
                 int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
                 if ((lo < 0) || (hi < lo) || (hi > p.T)) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);

@@ -70,7 +70,7 @@ def test_host_side_argument_checks(lib):
     assert _prefill(lib, binding, _layer(binding, A=0), ok_cache) == INVALID
     assert _prefill(lib, binding, _layer(binding, flags=2 | 4), ok_cache) == INVALID
     assert _prefill(lib, binding, ok_layer, ok_cache, x=None) == INVALID
-    assert _prefill(lib, binding, ok_layer, ok_cache, cu=None) == INVALID
+    assert _prefill(lib, binding, ok_layer, ok_cache, cu=None, n_seq=2) == INVALID   # offsets may be left out for one sequence only
     assert _prefill(lib, binding, ok_layer, ok_cache, ldx=32) == INVALID          # stride shorter than a row
     assert _prefill(lib, binding, ok_layer, ok_cache, x=0x100004) == MISALIGNED
     assert _prefill(lib, binding, ok_layer, ok_cache, ldb=18) == MISALIGNED       # 72-byte rows

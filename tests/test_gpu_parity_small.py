@@ -115,6 +115,28 @@ def test_prefill_in_place_slots_and_strided_views(act):
     assert_close(ref[0], o[0], TOL[act], "out")
 
 
+@pytest.mark.parametrize("chunk_len", [0, 48])
+def test_single_sequence_without_offsets_is_the_same_call(chunk_len):
+    """cu_seqlens = NULL with one sequence means rows 0..T-1: bit for bit what cu_seqlens = [0, T] gives."""
+    cfg = parity.small_config(264, "bf16", 1)
+    prob = parity.make_problem(cfg, [301], conv_bias=True, general_A=True)
+    tdt = torch.bfloat16
+    lay = upload_layer(prob.params, "bf16", md.MDRAFT_DT_SOFTPLUS)
+    dev = [to_device(a, tdt) for a in (prob.x, prob.z, prob.dt, prob.B, prob.C)]
+    res = []
+    for cu in (i32([0, 301]), None):
+        cache = md.StateCache(1, 1, 264, act=tdt)
+        out = torch.full((301, 264), float("nan"), dtype=tdt, device="cuda")
+        ws = torch.empty(max(256, md.mdraft_prefill_workspace_bytes(lay, 301, 1, 301, chunk_len)), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        md.mdraft_conv_scan_prefill(lay, cache, 0, *dev, out, cu, 301, None, i32([0]), ws, chunk_len, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        res.append((out.clone(), cache.ssm.clone(), cache.conv.clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+
+
 @pytest.mark.parametrize("act", ["f32", "bf16"])
 def test_prefill_chunking_is_only_a_schedule(act):
     """Different chunk lengths (including no chunking) agree with each other far inside the tolerance."""
