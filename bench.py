@@ -368,28 +368,62 @@ def run_ours(args):
         raise RuntimeError("device status bits set in the batched tree leg")
     clocks = sampler.stop()
 
-    # ---- end to end: pinned host inputs -> device -> the captured step -> outputs back to the host, every step
+    # ---- end to end: pinned host inputs -> device -> the path -> outputs back to the host, every step, through the
+    # public calls with their stream argument: three streams, so that layer l+1's inputs travel while layer l computes
+    # and layer l-1's outputs leave.  (The launches are eager here: each layer's calls wait on that layer's copy.)
+    s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(NL)]
+    ev_comp = [torch.cuda.Event() for _ in range(NL)]
+    ev_out = [torch.cuda.Event() for _ in range(NL)]
+    e2e_state = {"first": True}
+
     def e2e_step():
+        first = e2e_state["first"]
         for l in range(NL):
-            for d_t, h_t in zip(dev_pre[l], host_pre[l]):
-                d_t.copy_(h_t, non_blocking=True)
-            for d_t, h_t in zip(dev_node[l], host_node[l]):
-                d_t.copy_(h_t, non_blocking=True)
-        g_step.replay()
-        for l in range(NL):
-            host_out_pre[l].copy_(out_pre[l], non_blocking=True)
-            host_out_node[l].copy_(out_node[l], non_blocking=True)
+            with torch.cuda.stream(s_in):
+                if not first:
+                    s_in.wait_event(ev_comp[l])      # the previous step has finished reading this layer's inputs
+                for d_t, h_t in zip(dev_pre[l] + dev_node[l], host_pre[l] + host_node[l]):
+                    d_t.copy_(h_t, non_blocking=True)
+                ev_in[l].record(s_in)
+            with torch.cuda.stream(s_comp):
+                s_comp.wait_event(ev_in[l])
+                if not first:
+                    s_comp.wait_event(ev_out[l])     # the previous step's outputs of this layer have left
+                stack.prefill(dev_pre, out_pre, cu, T, None, slot0, s_comp, None, [l])
+                stack.tree_round(dev_node, out_node, parent_slot, node_slot, levels, s_comp, [l])
+                ev_comp[l].record(s_comp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_comp[l])
+                host_out_pre[l].copy_(out_pre[l], non_blocking=True)
+                host_out_node[l].copy_(out_node[l], non_blocking=True)
+                ev_out[l].record(s_out)
+        with torch.cuda.stream(s_comp):
+            stack.commit(acc_src, slot0, s_comp)
+        e2e_state["first"] = False
+
+    def e2e_join():
+        cur = torch.cuda.current_stream()
+        done = torch.cuda.Event()
+        for st in (s_in, s_comp, s_out):
+            done.record(st)
+            cur.wait_event(done)
 
     Ke = min(K, 5)
     for _ in range(2):
         e2e_step()
+    e2e_join()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
+    for st in (s_in, s_comp, s_out):
+        st.wait_event(e0)
     for _ in range(Ke):
         e2e_step()
+    e2e_join()
     e1.record()
     barrier()
+    stack.check_status()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / Ke
     h2d = sum(t.numel() * t.element_size() for l in range(NL) for t in host_pre[l] + host_node[l])
     d2h = sum(t.numel() * t.element_size() for l in range(NL) for t in (host_out_pre[l], host_out_node[l]))
