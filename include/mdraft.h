@@ -232,6 +232,34 @@ int mdraft_state_commit(const mdraft_cache *cache, int32_t d_inner, int32_t d_st
 int mdraft_classify_A(const float *A, int32_t d_inner, int32_t d_state, int32_t *scratch,
                       int32_t *is_powers, int32_t *is_nonpositive, void *stream);
 
+/*
+ * Test-time tree search (paper Section 4.2, Eq. 1-2 and Appendix A.4).  Each drafting round is a round of a
+ * multi-armed bandit whose K arms are preset tree configurations; the policy is UCB:
+ *
+ *     k* = argmax_k  mean_k + lambda_ucb * sqrt( 2 ln t / n_k )                                   (Eq. 1)
+ *     r  = -( 1 / N_accept + lambda_gamma * gamma / N_accept )    for the arm that was played      (Eq. 2)
+ *
+ * with t the round about to be played (from 1), n_k how often arm k was played, mean_k = reward_sum[k] / n_k the
+ * running mean of its rewards (the paper's "cumulative reward mean"), gamma the draft length (levels) of the played
+ * tree and N_accept >= 1 the tokens the round produced.  An arm that was never played is chosen first (lowest
+ * index first); ties go to the lowest index.  HOST code and HOST pointers throughout: the caller owns and zero-
+ * initialises reward_sum[n_arms], count[n_arms] and round; nothing here touches a GPU.
+ * Errors: NULL pointers, n_arms <= 0, arm out of range, draft_len < 1 or n_accept < 1 -> MDRAFT_ERR_INVALID_ARG.
+ */
+typedef struct {
+    int32_t n_arms;
+    int32_t reserved;
+    int64_t round;          /* rounds played so far */
+    double lambda_ucb;      /* exploration weight   */
+    double lambda_gamma;    /* drafter / target time per token (weight of the draft-length penalty) */
+    double *reward_sum;     /* HOST, n_arms */
+    int64_t *count;         /* HOST, n_arms */
+} mdraft_ucb;
+
+double mdraft_ucb_reward(double lambda_gamma, int32_t draft_len, int32_t n_accept);
+int mdraft_ucb_select(const mdraft_ucb *bandit, int32_t *arm);
+int mdraft_ucb_update(mdraft_ucb *bandit, int32_t arm, int32_t draft_len, int32_t n_accept);
+
 const char *mdraft_status_string(int status);
 
 /* Library version: major*10000 + minor*100 + patch. */

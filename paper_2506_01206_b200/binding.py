@@ -26,6 +26,7 @@ MDRAFT_DEV_BAD_SLOT, MDRAFT_DEV_BAD_SEQLENS, MDRAFT_DEV_WAIT_EXPIRED = 1, 2, 4
 EXPORTS = (
     "mdraft_prefill_workspace_bytes", "mdraft_conv_scan_prefill", "mdraft_conv_scan_prefill_noalloc", "mdraft_tree_step",
     "mdraft_state_commit", "mdraft_classify_A", "mdraft_status_string", "mdraft_version",
+    "mdraft_ucb_reward", "mdraft_ucb_select", "mdraft_ucb_update",
 )
 
 
@@ -51,6 +52,11 @@ class _Cache(C.Structure):
 class _PrefillOpts(C.Structure):
     _fields_ = [("chunk_len", C.c_int32), ("reserved", C.c_int32 * 3),
                 ("event_after_chunk_state", C.c_void_p), ("event_after_carry_scan", C.c_void_p)]
+
+
+class _Ucb(C.Structure):
+    _fields_ = [("n_arms", C.c_int32), ("reserved", C.c_int32), ("round", C.c_int64), ("lambda_ucb", C.c_double),
+                ("lambda_gamma", C.c_double), ("reward_sum", C.POINTER(C.c_double)), ("count", C.POINTER(C.c_int64))]
 
 
 _lib = None
@@ -89,6 +95,12 @@ def load_library(path: Optional[str] = None):
     lib.mdraft_state_commit.argtypes = [C.POINTER(_Cache), i32, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.mdraft_classify_A.restype = C.c_int
     lib.mdraft_classify_A.argtypes = [vp, i32, i32, vp, C.POINTER(i32), C.POINTER(i32), vp]
+    lib.mdraft_ucb_reward.restype = C.c_double
+    lib.mdraft_ucb_reward.argtypes = [C.c_double, i32, i32]
+    lib.mdraft_ucb_select.restype = C.c_int
+    lib.mdraft_ucb_select.argtypes = [C.POINTER(_Ucb), C.POINTER(i32)]
+    lib.mdraft_ucb_update.restype = C.c_int
+    lib.mdraft_ucb_update.argtypes = [C.POINTER(_Ucb), i32, i32, i32]
     if path is None:
         _lib = lib
     return lib
@@ -306,3 +318,40 @@ def mdraft_classify_A(A: torch.Tensor, stream=None):
     if rc != 0:
         raise MdraftError(rc, "mdraft_classify_A")
     return bool(a.value), bool(b.value)
+
+
+class UcbBandit:
+    """Arm statistics of the tree-configuration bandit, owned here, updated by the library (host code, no GPU)."""
+
+    def __init__(self, n_arms: int, lambda_ucb: float, lambda_gamma: float):
+        self._sum = (C.c_double * n_arms)()
+        self._cnt = (C.c_int64 * n_arms)()
+        self._c = _Ucb(int(n_arms), 0, 0, float(lambda_ucb), float(lambda_gamma), self._sum, self._cnt)
+
+    def mdraft_ucb_select(self) -> int:
+        arm = C.c_int32(-1)
+        rc = load_library().mdraft_ucb_select(C.byref(self._c), C.byref(arm))
+        if rc != 0:
+            raise MdraftError(rc, "mdraft_ucb_select")
+        return int(arm.value)
+
+    def mdraft_ucb_update(self, arm: int, draft_len: int, n_accept: int) -> None:
+        rc = load_library().mdraft_ucb_update(C.byref(self._c), int(arm), int(draft_len), int(n_accept))
+        if rc != 0:
+            raise MdraftError(rc, "mdraft_ucb_update")
+
+    @property
+    def reward_sum(self):
+        return list(self._sum)
+
+    @property
+    def count(self):
+        return list(self._cnt)
+
+    @property
+    def round(self) -> int:
+        return int(self._c.round)
+
+
+def mdraft_ucb_reward(lambda_gamma: float, draft_len: int, n_accept: int) -> float:
+    return float(load_library().mdraft_ucb_reward(float(lambda_gamma), int(draft_len), int(n_accept)))

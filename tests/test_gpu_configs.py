@@ -54,10 +54,12 @@ class Drafting:
         self.cfg, self.lay, self.olay, self.cache, self.li, self.S, self.watch, self.status = cfg, lay, olay, cache, layer_index, S, watch, status
         self.tdt = torch_act(cfg.act)
 
-    def round(self, rnd, committed):
-        """committed: {s: (conv (3,D), h (D,N))} oracle-side states of the watched sequences; updated in place."""
+    def round(self, rnd, committed, trees=None, accepted=None):
+        """committed: {s: (conv (3,D), h (D,N))} oracle-side states of the watched sequences; updated in place.
+        trees / accepted default to the configuration's own trees and seeded accepted nodes."""
         cfg, S = self.cfg, self.S
-        trees = [gen.config_tree(cfg, rnd, s) for s in range(S)]
+        if trees is None:
+            trees = [gen.config_tree(cfg, rnd, s) for s in range(S)]
         off = np.cumsum([0] + [t.n_nodes for t in trees])
         M = int(off[-1])
         x, z, dt, B, C = gen.node_inputs(cfg, self.li, rnd, M)          # rows in sequence-major order
@@ -76,7 +78,8 @@ class Drafting:
         dev = [to_device(a[order], self.tdt) for a in (x, z, dt, B, C)]
         out = torch.full((M, cfg.d_inner), float("nan"), dtype=self.tdt, device="cuda")
         md.mdraft_tree_step(self.lay, self.cache, self.li, *dev, out, i32(parent), i32(nodes), lvl, self.status)
-        accepted = [gen.random_accepted_node(trees[s], cfg.seed, cfg.cid, rnd, s) for s in range(S)]
+        if accepted is None:
+            accepted = [gen.random_accepted_node(trees[s], cfg.seed, cfg.cid, rnd, s) for s in range(S)]
         g_out = np.empty((M, cfg.d_inner))
         g_out[order] = _f64(out)
         worst = 0.0
@@ -207,3 +210,40 @@ def test_config4_packed_batch_and_four_rounds():
     for rnd in range(cfg.rounds):
         d.round(rnd, committed)
     assert int(status.item()) == 0
+
+
+def test_tree_search_drives_changing_tree_shapes():
+    """Section 4.2 end to end on the device path: a UCB bandit picks one of the paper's three tree configurations per
+    round, a synthetic verifier accepts a prefix of a random root-to-leaf path, the accepted node is committed, and
+    every round's node outputs and states are checked against the oracle.  The library's bandit and the oracle's
+    must take the same decisions."""
+    from oracle import tree_search as ots
+    configs = [(3, 3, 2, 1), (3, 2, 2, 1, 1), (2, 2, 2, 1, 1, 1)]
+    cfg = gen.Config(2, "search", 1, 1536, 16, 4, "bf16", 1, (512, 512), "none", 12, 5)
+    p, lay, olay = _layer(cfg, 1)
+    L = cfg.context[0]
+    max_nodes = max(gen.paper_tree(c).n_nodes for c in configs)
+    cache = md.StateCache(1, 1 + max_nodes, cfg.d_inner, act=torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ins = gen.prefill_inputs(cfg, 1, L)
+    _prefill(cfg, lay, cache, 0, ins, np.array([0, L]), [0], status)
+    _, o_conv, o_h = oracle.prefill(olay, *ins)
+    committed = {0: (o_conv[0], o_h[0])}
+    d = Drafting(cfg, lay, olay, cache, 0, 1, [0], status)
+    lib_b, ora_b = md.UcbBandit(3, 1.0, 0.05), ots.Bandit(3, 1.0, 0.05)
+    g = np.random.default_rng(3)
+    played = []
+    for rnd in range(cfg.rounds):
+        k = lib_b.mdraft_ucb_select()
+        assert k == ora_b.select()
+        tree = gen.paper_tree(configs[k])
+        ch, v, n_acc = tree.children(), 0, 1          # the root is the last verified token; walk down while accepted
+        while ch[v] and g.random() < 0.6:
+            v = ch[v][int(g.integers(0, len(ch[v])))]
+            n_acc += 1
+        d.round(rnd, committed, trees=[tree], accepted=[v])
+        lib_b.mdraft_ucb_update(k, len(configs[k]), n_acc)
+        ora_b.update(k, len(configs[k]), n_acc)
+        played.append(k)
+    assert int(status.item()) == 0
+    assert set(played[:3]) == {0, 1, 2} and lib_b.count == ora_b.n and lib_b.reward_sum == ora_b.r_sum
