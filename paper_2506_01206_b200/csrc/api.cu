@@ -75,9 +75,11 @@ struct PrefillPlan {
 };
 
 // Chunk length: split the token axis until every SM holds kBlocksPerSm blocks of kPrefillThreads channels (one
-// resident wave, no tail), but never into chunks shorter than kMinChunk tokens (per-chunk set-up would dominate) nor
-// longer than kMaxChunk (a batch of uneven sequences then still balances across SMs).
-constexpr int kBlocksPerSm = 4, kMinChunk = 32, kMaxChunk = 1024;
+// resident wave, no tail), but never into chunks shorter than kMinChunk tokens (per-chunk set-up would dominate).
+// When one wave would need chunks longer than kOneWaveMax tokens (long or batched contexts), several waves of short
+// chunks do better: blocks are then handed out as SMs free up, which evens out uneven sequences and keeps every SM
+// busy to the end (measured: 32768 tokens 404 -> 367 us, 32 packed sequences of 1k-8k tokens 1607 -> 1512 us).
+constexpr int kBlocksPerSm = 4, kMinChunk = 32, kOneWaveMax = 256, kManyWavesChunk = 128, kManyWavesChunkBatched = 256;
 
 PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen, const mdraft_prefill_opts* opts) {
     PrefillPlan pl;
@@ -90,7 +92,7 @@ PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen
         if (want < 1) want = 1;
         Lc = (T + want - 1) / want;
         if (Lc < kMinChunk) Lc = kMinChunk;
-        if (Lc > kMaxChunk) Lc = kMaxChunk;
+        if (Lc > kOneWaveMax) Lc = n_seq > 1 ? kManyWavesChunkBatched : kManyWavesChunk;
     }
     pl.chunked = Lc < max_seqlen;
     if (!pl.chunked) {
