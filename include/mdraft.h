@@ -114,7 +114,8 @@ typedef struct {
 /* Optional tuning and profiling hooks for the prefill; pass NULL for the defaults. */
 typedef struct {
     int32_t chunk_len;      /* tokens per scan chunk; 0 = chosen from the problem size; otherwise >= 4   */
-    int32_t reserved[3];    /* must be 0 */
+    int32_t block_channels; /* channels per thread block: 0 = chosen from the problem size, else 128 or 512 */
+    int32_t reserved[2];    /* must be 0 */
     void *event_after_chunk_state;  /* cudaEvent_t or NULL: recorded on `stream` after the chunk-summary kernel  */
     void *event_after_carry_scan;   /* cudaEvent_t or NULL: recorded after the carry scan, before the main scan  */
 } mdraft_prefill_opts;

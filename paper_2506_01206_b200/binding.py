@@ -50,7 +50,7 @@ class _Cache(C.Structure):
 
 
 class _PrefillOpts(C.Structure):
-    _fields_ = [("chunk_len", C.c_int32), ("reserved", C.c_int32 * 3),
+    _fields_ = [("chunk_len", C.c_int32), ("block_channels", C.c_int32), ("reserved", C.c_int32 * 2),
                 ("event_after_chunk_state", C.c_void_p), ("event_after_carry_scan", C.c_void_p)]
 
 
@@ -195,11 +195,16 @@ class StateCache:
         return self.ssm.numel() * 4 + self.conv.numel() * self.conv.element_size()
 
 
-def _opts(chunk_len: int, phase_events=None):
-    if not chunk_len and phase_events is None:
+def _opts(chunk_len, phase_events=None):
+    """chunk_len: tokens per chunk (0 = library's plan), or a pair (chunk_len, block_channels)."""
+    block_channels = 0
+    if isinstance(chunk_len, (tuple, list)):
+        chunk_len, block_channels = chunk_len
+    if not chunk_len and not block_channels and phase_events is None:
         return None
     o = _PrefillOpts()
     o.chunk_len = int(chunk_len)
+    o.block_channels = int(block_channels)
     if phase_events is not None:  # two torch.cuda.Event objects (already created with enable_timing=True)
         o.event_after_chunk_state = phase_events[0].cuda_event
         o.event_after_carry_scan = phase_events[1].cuda_event

@@ -71,6 +71,7 @@ struct PrefillPlan {
     int chunk_len;       // tokens per chunk (INT_MAX/2 when every sequence is one chunk)
     int n_chunks_bound;  // upper bound on the number of chunks
     bool chunked;
+    bool wide;           // 512-channel blocks (one per SM) instead of 128-channel blocks
     size_t off_q, off_sd, off_h0, off_conv, bytes;
 };
 
@@ -83,17 +84,29 @@ constexpr int kBlocksPerSm = 4, kMinChunk = 32, kOneWaveMax = 256, kManyWavesChu
 
 PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen, const mdraft_prefill_opts* opts) {
     PrefillPlan pl;
+    const int D = L->d_inner;
+    const int wide_cols = kPrefillThreads * kPrefillWideBoxes;
+    const int ch_blocks = (D + kPrefillThreads - 1) / kPrefillThreads;
+    const int ch_blocks_wide = (D + wide_cols - 1) / wide_cols;
+    const int forced = opts ? opts->block_channels : 0;
+    // Wide blocks pay off when they fill the machine in one wave: every SM then runs ONE block whose 16 channel warps
+    // advance together and finish together (four narrow blocks per SM finish one after another and leave the SM to
+    // the last of them).  They need the channel count to (nearly) fill whole 512-channel blocks.
+    bool wide = forced == wide_cols || (forced == 0 && (int64_t)ch_blocks_wide * wide_cols * 9 <= (int64_t)D * 10);
     int Lc;
     if (opts && opts->chunk_len > 0) {
         Lc = opts->chunk_len < 4 ? 4 : opts->chunk_len;
     } else {
-        const int ch_blocks = (L->d_inner + kPrefillThreads - 1) / kPrefillThreads;
-        int want = kSmCount * kBlocksPerSm / ch_blocks;
+        int want = wide ? kSmCount / ch_blocks_wide : kSmCount * kBlocksPerSm / ch_blocks;
         if (want < 1) want = 1;
         Lc = (T + want - 1) / want;
         if (Lc < kMinChunk) Lc = kMinChunk;
-        if (Lc > kOneWaveMax) Lc = n_seq > 1 ? kManyWavesChunkBatched : kManyWavesChunk;
+        if (Lc > kOneWaveMax) {  // several waves: narrow blocks, four to an SM, so that a new block's set-up hides behind the others
+            Lc = n_seq > 1 ? kManyWavesChunkBatched : kManyWavesChunk;
+            if (forced == 0) wide = false;
+        }
     }
+    pl.wide = wide;
     pl.chunked = Lc < max_seqlen;
     if (!pl.chunked) {
         pl.chunk_len = INT_MAX / 2;
@@ -104,12 +117,12 @@ PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen
     }
     pl.chunk_len = Lc;
     pl.n_chunks_bound = n_seq + T / Lc;
-    const size_t D = (size_t)L->d_inner;
+    const size_t Dz = (size_t)D;
     pl.off_q = 0;
-    pl.off_sd = align_up(pl.off_q + (size_t)pl.n_chunks_bound * D * kN * sizeof(float), 256);
-    pl.off_h0 = align_up(pl.off_sd + (size_t)pl.n_chunks_bound * D * sizeof(float), 256);
-    pl.off_conv = align_up(pl.off_h0 + (size_t)n_seq * D * kN * sizeof(float), 256);
-    pl.bytes = align_up(pl.off_conv + (size_t)n_seq * (kW - 1) * D * elem_size(L->act), 256);
+    pl.off_sd = align_up(pl.off_q + (size_t)pl.n_chunks_bound * Dz * kN * sizeof(float), 256);
+    pl.off_h0 = align_up(pl.off_sd + (size_t)pl.n_chunks_bound * Dz * sizeof(float), 256);
+    pl.off_conv = align_up(pl.off_h0 + (size_t)n_seq * Dz * kN * sizeof(float), 256);
+    pl.bytes = align_up(pl.off_conv + (size_t)n_seq * (kW - 1) * Dz * elem_size(L->act), 256);
     return pl;
 }
 
@@ -187,8 +200,10 @@ int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cach
     if (total_tokens < 0 || n_seq < 0 || max_seqlen < 0) return MDRAFT_ERR_INVALID_ARG;
     if (opts) {
         if (opts->chunk_len < 0) return MDRAFT_ERR_INVALID_ARG;
-        for (int i = 0; i < 3; ++i)
+        for (int i = 0; i < 2; ++i)
             if (opts->reserved[i]) return MDRAFT_ERR_INVALID_ARG;
+        if (opts->block_channels != 0 && opts->block_channels != kPrefillThreads && opts->block_channels != kPrefillThreads * kPrefillWideBoxes)
+            return MDRAFT_ERR_INVALID_ARG;
     }
     const bool needs_pool = init_slot || final_slot;
     if (needs_pool || cache) {
@@ -237,7 +252,7 @@ int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cach
         !encode_matrix(&maps.B, have_rows ? B : nullptr, act, total_tokens, kN, ldb, kN) ||
         !encode_matrix(&maps.C, have_rows ? C : nullptr, act, total_tokens, kN, ldc, kN))
         return MDRAFT_ERR_CUDA;
-    cudaError_t e = launch_prefill(a, maps, act, pl.chunked, static_cast<cudaStream_t>(stream));
+    cudaError_t e = launch_prefill(a, maps, act, pl.chunked, pl.wide, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? MDRAFT_OK : MDRAFT_ERR_CUDA;
 }
 

@@ -14,12 +14,12 @@
 // A call in which every sequence fits one chunk runs the output pass only.
 //
 // Data movement.  One thread owns one channel and keeps its 16 state entries in registers as 8 packed pairs
-// (fma.rn.f32x2 / mul.rn.f32x2: one instruction per two entries).  A block of 128 channels walks its chunk in
+// (fma.rn.f32x2 / mul.rn.f32x2: one instruction per two entries).  A block of 128 or 512 channels walks its chunk in
 // tiles of 16 (bf16) or 8 (fp32) tokens; the x / dt / z boxes (tile x 128 channels) and the B / C boxes of a tile
 // are brought into a ring of shared-memory stages by TMA (cp.async.bulk.tensor, one instruction per matrix and
-// tile, completion counted on an mbarrier), two tiles ahead of the arithmetic.  The block is warp-specialised: a fifth warp queues the copies,
-// widens each landed B / C tile to fp32 (read afterwards as 128-bit broadcasts) and hands it to the four
-// channel warps through a "ready" mbarrier; each channel warp releases a stage through an "empty" mbarrier
+// tile, completion counted on an mbarrier), two tiles ahead of the arithmetic.  The block is warp-specialised: one extra
+// warp queues the copies, widens each landed B / C tile to fp32 (read afterwards as 128-bit broadcasts) and hands it
+// to the 4 or 16 channel warps through a "ready" mbarrier; each channel warp releases a stage through an "empty" mbarrier
 // when it is done, so the channel warps never wait for one another.  Every wait on an mbarrier is bounded: if
 // it runs out, the warp raises MDRAFT_DEV_WAIT_EXPIRED and stops; the copy warp first gives the copies it still
 // has in flight a bounded chance to land (they target this block's shared memory).
@@ -30,13 +30,20 @@ namespace mdraft {
 
 namespace {
 
-constexpr int kCB = kPrefillThreads;    // channels per block, one thread each
-constexpr int kBlockThreads = kCB + 32; // plus the copy warp
+constexpr int kBoxCols = kPrefillThreads;  // channels of one TMA box (and of one group of four channel warps)
 constexpr int kStages = 3;              // shared-memory ring depth
-constexpr int kTileBytes = 4096;        // one staged x / dt / z tile: kTT rows of kCB activations
+constexpr int kTileBytes = 4096;        // one staged x / dt / z box: kTT rows of kBoxCols activations
 constexpr int kBCBytes = 512;           // one staged B or C tile: kTT rows of 16 activations
-constexpr int kStageBytes = 3 * kTileBytes + 2 * kBCBytes;
-constexpr int kOffX = 0, kOffDt = kTileBytes, kOffZ = 2 * kTileBytes, kOffB = 3 * kTileBytes, kOffC = 3 * kTileBytes + kBCBytes;
+// A block covers SUB boxes of channels (SUB = 1: 128 channels, 4 channel warps; SUB = 4: 512 channels, 16 channel
+// warps that share the block's B / C tiles and advance tile by tile together).  Stage layout: x boxes, dt boxes,
+// z boxes, B, C.
+__host__ __device__ constexpr int stage_bytes(int sub) { return 3 * sub * kTileBytes + 2 * kBCBytes; }
+__host__ __device__ constexpr int off_x(int) { return 0; }
+__host__ __device__ constexpr int off_dt(int sub) { return sub * kTileBytes; }
+__host__ __device__ constexpr int off_z(int sub) { return 2 * sub * kTileBytes; }
+__host__ __device__ constexpr int off_b(int sub) { return 3 * sub * kTileBytes; }
+__host__ __device__ constexpr int off_c(int sub) { return 3 * sub * kTileBytes + kBCBytes; }
+__host__ __device__ constexpr int smem_bytes(int sub) { return kStages * (stage_bytes(sub) + 2 * kBCBytes * 2); }  // + fp32 B, C
 constexpr int GRP = 4;                  // tokens whose state-independent part is computed together (measured: 2 % faster than one by one)
 constexpr uint32_t kSpinLimit = 1u << 20;  // polls of one mbarrier before the block gives up
 
@@ -317,25 +324,37 @@ __device__ __forceinline__ void load_window(float* win, const AT* x, int64_t ldx
     }
 }
 
-// One lane queues the copies of one tile: a box per matrix.  `mask`: bit 0 = dt, bit 1 = z, bit 2 = B, bit 3 = C
-// (x is always copied).  Every box is full size whatever part of it lies inside the matrix.
-__device__ __forceinline__ void issue_tile(unsigned char* stage, uint64_t* bar, const PrefillMaps& m, int t, int d0, uint32_t mask) {
+// One lane queues the copies of one tile: per matrix one box for every 128 channels of the block that exist.
+// `mask`: bit 0 = dt, bit 1 = z, bit 2 = B, bit 3 = C (x is always copied).  Every box is full size whatever part
+// of it lies inside the matrix.
+template <int SUB>
+__device__ __forceinline__ void issue_tile(unsigned char* stage, uint64_t* bar, const PrefillMaps& m, int t, int d0, int D, uint32_t mask) {
     const uint32_t n_wide = 1u + (mask & 1u) + ((mask >> 1) & 1u), n_bc = ((mask >> 2) & 1u) + ((mask >> 3) & 1u);
-    mbar_expect_tx(bar, n_wide * kTileBytes + n_bc * kBCBytes);
-    tma_box(stage + kOffX, &m.x, d0, t, bar);
-    if (mask & 1u) tma_box(stage + kOffDt, &m.dt, d0, t, bar);
-    if (mask & 2u) tma_box(stage + kOffZ, &m.z, d0, t, bar);
-    if (mask & 4u) tma_box(stage + kOffB, &m.B, 0, t, bar);
-    if (mask & 8u) tma_box(stage + kOffC, &m.C, 0, t, bar);
+    const uint32_t subs = (uint32_t)min(SUB, (D - d0 + kBoxCols - 1) / kBoxCols);
+    mbar_expect_tx(bar, subs * n_wide * kTileBytes + n_bc * kBCBytes);
+#pragma unroll
+    for (int sb = 0; sb < SUB; ++sb) {
+        if (sb < (int)subs) {
+            const int c = d0 + sb * kBoxCols;
+            tma_box(stage + off_x(SUB) + sb * kTileBytes, &m.x, c, t, bar);
+            if (mask & 1u) tma_box(stage + off_dt(SUB) + sb * kTileBytes, &m.dt, c, t, bar);
+            if (mask & 2u) tma_box(stage + off_z(SUB) + sb * kTileBytes, &m.z, c, t, bar);
+        }
+    }
+    if (mask & 4u) tma_box(stage + off_b(SUB), &m.B, 0, t, bar);
+    if (mask & 8u) tma_box(stage + off_c(SUB), &m.C, 0, t, bar);
 }
 
 // ---------------------------------------------------------------------------------------------------
-template <typename AT, bool kPow, bool kOut, bool kFast>
-__global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs p, const __grid_constant__ PrefillMaps maps) {
+template <typename AT, int SUB, bool kPow, bool kOut, bool kFast>
+__global__ void __launch_bounds__(SUB * kBoxCols + 32) chunk_kernel(const PrefillArgs p, const __grid_constant__ PrefillMaps maps) {
     constexpr int TT = TileTokens<AT>::v;
-    __shared__ __align__(128) unsigned char s_stage[kStages][kStageBytes];
-    __shared__ __align__(16) float sBf[kStages][TT][kN];
-    __shared__ __align__(16) float sCf[kStages][TT][kN];
+    constexpr int kCB = SUB * kBoxCols;          // channels per block, one thread each
+    constexpr int kStageBytes = stage_bytes(SUB);
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    unsigned char (*s_stage)[kStageBytes] = reinterpret_cast<unsigned char (*)[kStageBytes]>(s_dyn);
+    float (*sBf)[TT][kN] = reinterpret_cast<float (*)[TT][kN]>(s_dyn + kStages * kStageBytes);
+    float (*sCf)[TT][kN] = reinterpret_cast<float (*)[TT][kN]>(s_dyn + kStages * kStageBytes + kStages * TT * kN * 4);
     __shared__ __align__(8) uint64_t bar_raw[kStages];    // copies of a tile have landed (transaction count)
     __shared__ __align__(8) uint64_t bar_ready[kStages];  // ... and its B / C are widened: channel warps may start
     __shared__ __align__(8) uint64_t bar_empty[kStages];  // all channel warps are done with the stage
@@ -429,7 +448,7 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
     const bool want_c = kOut && !conv_only;
     const int pre = min(kStages - 1, ntiles);
     if (copy_warp && lane == 0)  // the first tiles go out before anything else is looked up
-        for (int j = 0; j < pre; ++j) issue_tile(s_stage[j], &bar_raw[j], maps, ci.t0 + j * TT, d0, mask);
+        for (int j = 0; j < pre; ++j) issue_tile<SUB>(s_stage[j], &bar_raw[j], maps, ci.t0 + j * TT, d0, D, mask);
 
     const int islot = load_slot(p.init_slot, ci.seq);
     const int fslot = load_slot(p.final_slot, ci.seq);
@@ -452,8 +471,8 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
             landed = j + 1;
             if (!conv_only) {
                 const int rows = min(TT, ci.t1 - (ci.t0 + j * TT));
-                const AT* rb = reinterpret_cast<const AT*>(s_stage[s] + kOffB);
-                const AT* rc = reinterpret_cast<const AT*>(s_stage[s] + kOffC);
+                const AT* rb = reinterpret_cast<const AT*>(s_stage[s] + off_b(SUB));
+                const AT* rc = reinterpret_cast<const AT*>(s_stage[s] + off_c(SUB));
                 for (int i = lane; i < rows * kN; i += 32) {
                     (&sBf[s][0][0])[i] = Act<AT>::to_f32(rb[i]);
                     if (want_c) (&sCf[s][0][0])[i] = Act<AT>::to_f32(rc[i]);
@@ -465,7 +484,7 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
             if (nxt < ntiles) {
                 if (nxt >= kStages) ok = mbar_wait_bounded(&bar_empty[nxt % kStages], (uint32_t)(nxt / kStages - 1) & 1u);
                 if (!ok) break;
-                if (lane == 0) issue_tile(s_stage[nxt % kStages], &bar_raw[nxt % kStages], maps, ci.t0 + nxt * TT, d0, mask);
+                if (lane == 0) issue_tile<SUB>(s_stage[nxt % kStages], &bar_raw[nxt % kStages], maps, ci.t0 + nxt * TT, d0, D, mask);
                 queued = nxt + 1;
             }
         }
@@ -530,9 +549,10 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
         }
         if (live) {
             const unsigned char* st = s_stage[s];
-            const AT* sx = reinterpret_cast<const AT*>(st + kOffX) + tid;
-            const AT* sdt = reinterpret_cast<const AT*>(st + kOffDt) + tid;
-            const AT* sz = reinterpret_cast<const AT*>(st + kOffZ) + tid;
+            const int box = (tid / kBoxCols) * kTileBytes, col = tid % kBoxCols;  // this thread's box of 128 channels and its column in it
+            const AT* sx = reinterpret_cast<const AT*>(st + off_x(SUB) + box) + col;
+            const AT* sdt = reinterpret_cast<const AT*>(st + off_dt(SUB) + box) + col;
+            const AT* sz = reinterpret_cast<const AT*>(st + off_z(SUB) + box) + col;
             AT* orow = out + (size_t)t * p.ldo + d;
             typedef typename ChannelScan<AT, kPow, kOut, kFast>::Pre Pre;
             int r = 0;
@@ -541,9 +561,9 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
                 float o[GRP];
 #pragma unroll
                 for (int g = 0; g < GRP; ++g) {
-                    const float xv = Act<AT>::to_f32(sx[(r + g) * kCB]);
-                    const float dtv = conv_only ? 0.0f : Act<AT>::to_f32(sdt[(r + g) * kCB]);
-                    const float zv = want_c ? Act<AT>::to_f32(sz[(r + g) * kCB]) : 0.0f;
+                    const float xv = Act<AT>::to_f32(sx[(r + g) * kBoxCols]);
+                    const float dtv = conv_only ? 0.0f : Act<AT>::to_f32(sdt[(r + g) * kBoxCols]);
+                    const float zv = want_c ? Act<AT>::to_f32(sz[(r + g) * kBoxCols]) : 0.0f;
                     cs.pre(xv, zv, dtv, e[g]);
                 }
 #pragma unroll
@@ -555,9 +575,9 @@ __global__ void __launch_bounds__(kBlockThreads) chunk_kernel(const PrefillArgs 
             }
             for (; r < rows; ++r) {
                 Pre e;
-                const float xv = Act<AT>::to_f32(sx[r * kCB]);
-                const float dtv = conv_only ? 0.0f : Act<AT>::to_f32(sdt[r * kCB]);
-                const float zv = want_c ? Act<AT>::to_f32(sz[r * kCB]) : 0.0f;
+                const float xv = Act<AT>::to_f32(sx[r * kBoxCols]);
+                const float dtv = conv_only ? 0.0f : Act<AT>::to_f32(sdt[r * kBoxCols]);
+                const float zv = want_c ? Act<AT>::to_f32(sz[r * kBoxCols]) : 0.0f;
                 cs.pre(xv, zv, dtv, e);
                 const float o = cs.post(e, sBf[s][r], sCf[s][r]);
                 if (kOut) orow[(size_t)r * p.ldo] = Act<AT>::from_f32(o);
@@ -682,11 +702,11 @@ __global__ void __launch_bounds__(kCarryGroups * 32) carry_kernel(const PrefillA
 
 // Launch with programmatic stream serialisation: the kernel may begin before the one ahead of it has finished.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, cudaStream_t st, Args... args) {
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(threads);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -696,39 +716,53 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, cudaStr
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-template <typename AT, bool kPow, bool kFast>
+// The wide block needs more dynamic shared memory than a kernel gets by default; the limit is raised once per
+// kernel and device (a property of the loaded function, not an allocation).
+template <typename K>
+cudaError_t allow_smem(K kernel, int bytes) {
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+template <typename AT, int SUB, bool kPow, bool kFast>
 cudaError_t launch_typed(PrefillArgs p, const PrefillMaps& maps, bool chunked, cudaStream_t st) {
     const int D = p.L.d_inner;
+    constexpr int kCB = SUB * kBoxCols, kThreads = kCB + 32, kSmem = smem_bytes(SUB);
     dim3 grid((D + kCB - 1) / kCB, p.n_chunks_bound);
     const bool recur = !(p.L.flags & MDRAFT_CONV_ONLY);
     p.pdl_inputs_ready = chunked ? 1 : 0;  // the summary pass waits for the producer of the inputs on behalf of all three
     cudaError_t e = cudaSuccess;
-    if (chunked) e = launch_pdl(chunk_kernel<AT, kPow, false, kFast>, grid, kBlockThreads, st, p, maps);
+    if (chunked) {
+        if ((e = allow_smem(chunk_kernel<AT, SUB, kPow, false, kFast>, kSmem)) != cudaSuccess) return e;
+        e = launch_pdl(chunk_kernel<AT, SUB, kPow, false, kFast>, grid, kThreads, kSmem, st, p, maps);
+    }
     if (e != cudaSuccess) return e;
     if (p.ev_state) cudaEventRecord(p.ev_state, st);
     if (chunked && recur) {
         dim3 g2((D + 31) / 32, kN / 4, p.n_seq);
-        e = launch_pdl(carry_kernel, g2, kCarryGroups * 32, st, p);
+        e = launch_pdl(carry_kernel, g2, kCarryGroups * 32, 0, st, p);
         if (e != cudaSuccess) return e;
     }
     if (p.ev_carry) cudaEventRecord(p.ev_carry, st);
-    e = launch_pdl(chunk_kernel<AT, kPow, true, kFast>, grid, kBlockThreads, st, p, maps);
+    if ((e = allow_smem(chunk_kernel<AT, SUB, kPow, true, kFast>, kSmem)) != cudaSuccess) return e;
+    e = launch_pdl(chunk_kernel<AT, SUB, kPow, true, kFast>, grid, kThreads, kSmem, st, p, maps);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
-template <typename AT>
+template <typename AT, int SUB>
 cudaError_t launch_act(const PrefillArgs& p, const PrefillMaps& maps, bool chunked, cudaStream_t st) {
     const bool pow = p.L.flags & MDRAFT_A_POWERS;
     const bool fast = (p.L.flags & ~(uint32_t)MDRAFT_A_POWERS) == (uint32_t)MDRAFT_DT_SOFTPLUS;
-    if (fast) return pow ? launch_typed<AT, true, true>(p, maps, chunked, st) : launch_typed<AT, false, true>(p, maps, chunked, st);
-    return pow ? launch_typed<AT, true, false>(p, maps, chunked, st) : launch_typed<AT, false, false>(p, maps, chunked, st);
+    if (fast) return pow ? launch_typed<AT, SUB, true, true>(p, maps, chunked, st) : launch_typed<AT, SUB, false, true>(p, maps, chunked, st);
+    return pow ? launch_typed<AT, SUB, true, false>(p, maps, chunked, st) : launch_typed<AT, SUB, false, false>(p, maps, chunked, st);
 }
 
 }  // namespace
 
-cudaError_t launch_prefill(const PrefillArgs& p, const PrefillMaps& maps, int act, bool chunked, cudaStream_t st) {
-    return act == MDRAFT_F32 ? launch_act<float>(p, maps, chunked, st) : launch_act<__nv_bfloat16>(p, maps, chunked, st);
+cudaError_t launch_prefill(const PrefillArgs& p, const PrefillMaps& maps, int act, bool chunked, bool wide, cudaStream_t st) {
+    if (wide) return act == MDRAFT_F32 ? launch_act<float, kPrefillWideBoxes>(p, maps, chunked, st) : launch_act<__nv_bfloat16, kPrefillWideBoxes>(p, maps, chunked, st);
+    return act == MDRAFT_F32 ? launch_act<float, 1>(p, maps, chunked, st) : launch_act<__nv_bfloat16, 1>(p, maps, chunked, st);
 }
 
 }  // namespace mdraft

@@ -35,6 +35,9 @@ struct PrefillMaps {
     CUtensorMap x, dt, z, B, C;
 };
 
-cudaError_t launch_prefill(const PrefillArgs& p, const PrefillMaps& maps, int act, bool chunked, cudaStream_t st);
+constexpr int kPrefillWideBoxes = 4;  // a wide block covers 4 x kPrefillThreads channels with 16 channel warps
+
+// wide: one block of 512 channels per (channel block, chunk) instead of 128 — for plans that give every SM one block.
+cudaError_t launch_prefill(const PrefillArgs& p, const PrefillMaps& maps, int act, bool chunked, bool wide, cudaStream_t st);
 
 }  // namespace mdraft

@@ -85,7 +85,7 @@ def test_host_side_argument_checks(lib):
     assert need > 0 and need % 256 == 0
     assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(opts), ws=0x900000, ws_bytes=need - 1) == WORKSPACE
     assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(opts), ws=0x900010, ws_bytes=need) == MISALIGNED
-    bad = binding._PrefillOpts(); bad.chunk_len = 8; bad.reserved[2] = 1
+    bad = binding._PrefillOpts(); bad.chunk_len = 8; bad.reserved[1] = 1
     assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(bad)) == INVALID
     # nothing to do is fine and launches nothing
     assert _prefill(lib, binding, ok_layer, ok_cache, n_seq=0, T=0, cu=None) == 0

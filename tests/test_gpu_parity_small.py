@@ -115,6 +115,27 @@ def test_prefill_in_place_slots_and_strided_views(act):
     assert_close(ref[0], o[0], TOL[act], "out")
 
 
+@pytest.mark.parametrize("act,Dn,lens,chunk_len", [
+    ("bf16", 200, [333], 50),                    # two boxes of channels, the second one partly outside the matrix
+    ("f32", 264, [90, 17, 150], 32),             # three boxes, packed sequences
+    ("bf16", 1024, [40, 300, 7, 129], 37),       # two full wide blocks
+    ("bf16", 520, [260], 0),                     # a second wide block that holds 8 channels only; default chunk plan
+])
+def test_prefill_wide_and_narrow_blocks_agree_with_the_oracle(act, Dn, lens, chunk_len):
+    """Both block widths (128 channels with 4 channel warps, 512 channels with 16) against the oracle, forced through
+    the block_channels option, on channel counts that leave boxes partly or wholly empty."""
+    cfg = parity.small_config(Dn, act, len(lens))
+    prob = parity.make_problem(cfg, lens, conv_bias=True, general_A=True)
+    ci, hi = random_state(cfg, len(lens), 5)
+    flags = md.MDRAFT_DT_SOFTPLUS
+    o_out, o_conv, o_h = run_oracle_prefill(prob, flags, ci, hi)
+    for block_channels in (128, 512):
+        g_out, g_conv, g_h = run_gpu_prefill(prob, flags, (chunk_len, block_channels), ci, hi)
+        assert_close(g_out, o_out, TOL[act], f"out, {block_channels}-channel blocks")
+        assert_close(g_h, o_h, TOL_STATE, f"final SSM state, {block_channels}-channel blocks")
+        assert np.array_equal(g_conv, o_conv)
+
+
 @pytest.mark.parametrize("chunk_len", [0, 48])
 def test_single_sequence_without_offsets_is_the_same_call(chunk_len):
     """cu_seqlens = NULL with one sequence means rows 0..T-1: bit for bit what cu_seqlens = [0, T] gives."""
