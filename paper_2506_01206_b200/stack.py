@@ -62,3 +62,60 @@ class DrafterStack:
         s = int(self.status.item())
         if s:
             raise RuntimeError(f"device status bits set: {s:#x}")
+
+
+class RoundGraphCache:
+    """CUDA graphs of draft rounds, one per tree shape, replayed instead of re-launched.
+
+    The paper caches one CUDA graph per batch size of its drafter (Section 4.1, "Efficient cache utilization"); here
+    a graph covers a whole round — every level of every layer plus the commit — and is keyed by the tree's level
+    sizes, which is all the launch geometry depends on.  Everything a round reads lives in static device buffers owned
+    by this object (node inputs per layer, parent / node slots, the accepted node's slot), so a replay sees whatever
+    the caller last copied into them; the library's calls take their indices from device memory, which is what makes
+    one capture valid for every tree of that shape.
+    """
+
+    def __init__(self, stack: DrafterStack, max_nodes: int, seq_slot: int = 0):
+        self.stack = stack
+        dev, D, act = stack.status.device, stack.d_inner, stack.act
+        n = len(stack.layers)
+        self.x = [torch.zeros((max_nodes, D), dtype=act, device=dev) for _ in range(n)]
+        self.z = [torch.zeros((max_nodes, D), dtype=act, device=dev) for _ in range(n)]
+        self.dt = [torch.zeros((max_nodes, D), dtype=act, device=dev) for _ in range(n)]
+        self.B = [torch.zeros((max_nodes, 16), dtype=act, device=dev) for _ in range(n)]
+        self.C = [torch.zeros((max_nodes, 16), dtype=act, device=dev) for _ in range(n)]
+        self.out = [torch.zeros((max_nodes, D), dtype=act, device=dev) for _ in range(n)]
+        self.parent_slot = torch.zeros(max_nodes, dtype=torch.int32, device=dev)
+        self.node_slot = torch.zeros(max_nodes, dtype=torch.int32, device=dev)
+        self.accepted_slot = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.seq_slot = torch.full((1,), seq_slot, dtype=torch.int32, device=dev)
+        self.max_nodes = max_nodes
+        self._graphs = {}
+
+    def _launch(self, level_offsets) -> None:
+        m = level_offsets[-1]
+        ins = [(self.x[l][:m], self.z[l][:m], self.dt[l][:m], self.B[l][:m], self.C[l][:m]) for l in range(len(self.stack.layers))]
+        outs = [o[:m] for o in self.out]
+        self.stack.tree_round(ins, outs, self.parent_slot[:m], self.node_slot[:m], level_offsets)
+        self.stack.commit(self.accepted_slot, self.seq_slot)
+
+    def run(self, level_offsets: Sequence[int]) -> bool:
+        """Run one round (all levels, all layers, then the commit of `accepted_slot`) for a tree with these level
+        offsets.  Returns True when an existing graph was replayed, False when the shape was new and got captured."""
+        key = tuple(int(v) for v in level_offsets)
+        if key[-1] > self.max_nodes:
+            raise ValueError("tree larger than the buffers of this cache")
+        g = self._graphs.get(key)
+        if g is not None:
+            g.replay()
+            return True
+        self._launch(list(key))           # first use of a shape runs eagerly once (nothing new happens inside a capture)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self._launch(list(key))
+        self._graphs[key] = g
+        return False
+
+    def __len__(self) -> int:
+        return len(self._graphs)

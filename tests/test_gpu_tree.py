@@ -193,3 +193,47 @@ def test_tree_step_bad_slots_are_skipped_and_flagged():
     o = out.float().cpu().numpy()
     assert np.all(np.isnan(o[2])) and np.all(np.isnan(o[4])), "skipped nodes write nothing"
     assert np.all(np.isfinite(o[[0, 1, 3]]))
+
+
+def test_round_graph_cache_replays_what_eager_launches_compute():
+    """One captured graph per tree shape (the paper caches one per batch size, Section 4.1): a replay with new inputs,
+    new slot indices and another accepted node must give, bit for bit, what the same round gives launched eagerly."""
+    from paper_2506_01206_b200.stack import DrafterStack, RoundGraphCache
+    cfg = parity.small_config(264, "bf16")
+    n_layers = 3
+    params = [gen.layer_params(cfg, l, conv_bias=True, general_A=True) for l in range(n_layers)]
+    tdt = torch.bfloat16
+
+    def fresh_stack():
+        st = DrafterStack([upload_layer(p, "bf16") for p in params], 1 + 48, 16, 1, 16)
+        g = torch.Generator(device="cuda").manual_seed(7)
+        st.cache.ssm[:, 0] = torch.randn(st.cache.ssm[:, 0].shape, generator=g, device="cuda")
+        st.cache.conv[:, 0] = torch.randn(st.cache.conv[:, 0].shape, generator=g, device="cuda").to(tdt)
+        return st
+
+    shapes = [gen.paper_tree((3, 2, 2, 1, 1)), gen.paper_tree((2, 2, 2, 1, 1, 1)), gen.paper_tree((3, 2, 2, 1, 1))]
+    graph_stack, eager_stack = fresh_stack(), fresh_stack()
+    cache = RoundGraphCache(graph_stack, max_nodes=48)
+    replayed = []
+    for rnd, tree in enumerate(shapes):
+        M = tree.n_nodes
+        levels = [int(v) for v in tree.level_offsets]
+        parent = i32(np.where(tree.parents < 0, 0, tree.parents + 1))
+        nodes = i32(np.arange(M) + 1)
+        accepted = i32([1 + gen.random_accepted_node(tree, 0, 93, rnd)])
+        ins = [[to_device(a, tdt) for a in gen.node_inputs(cfg, l, rnd, M)] for l in range(n_layers)]
+        for l in range(n_layers):
+            for buf, a in zip((cache.x[l], cache.z[l], cache.dt[l], cache.B[l], cache.C[l]), ins[l]):
+                buf[:M].copy_(a)
+        cache.parent_slot[:M].copy_(parent); cache.node_slot[:M].copy_(nodes); cache.accepted_slot.copy_(accepted)
+        replayed.append(cache.run(levels))
+        outs = [torch.empty((M, 264), dtype=tdt, device="cuda") for _ in range(n_layers)]
+        eager_stack.tree_round(ins, outs, parent, nodes, levels)
+        eager_stack.commit(accepted, i32([0]))
+        torch.cuda.synchronize()
+        for l in range(n_layers):
+            assert torch.equal(cache.out[l][:M], outs[l])
+        assert torch.equal(graph_stack.cache.ssm.view(torch.int32), eager_stack.cache.ssm.view(torch.int32))
+        assert torch.equal(graph_stack.cache.conv.view(torch.int16), eager_stack.cache.conv.view(torch.int16))
+    assert replayed == [False, False, True] and len(cache) == 2
+    graph_stack.check_status(); eager_stack.check_status()
