@@ -70,7 +70,7 @@ class Workload:
     def node_inputs(self, l):
         return gen.node_inputs(self.cfg, l, 0, self.M)
 
-    # algorithmic bytes (see DESIGN.md): activations in/out + B,C + final state write
+    # algorithmic bytes: activations in/out + B,C + final state write
     def prefill_bytes_per_layer(self):
         D, N, T, es = self.cfg.d_inner, self.cfg.d_state, self.T, 2
         return 4 * es * T * D + 2 * N * es * T + D * N * 4 + 3 * D * es
@@ -183,7 +183,9 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------------------------- GPU leg
-ALU_LANE_OPS_PER_UNIT = 82      # fp32 lane-operations per token*channel of a single-pass prefill (derivation in the design doc)
+# fp32 lane-operations per token*channel of a single-pass prefill: conv 4 + SiLU 3 + softplus 5 + step*input 1 +
+# 16 states x (form the decay, decay*h, input*B, C*h) 64 + skip 1 + gate 4
+ALU_LANE_OPS_PER_UNIT = 82
 FP32_LANES_PER_SM, SM_COUNT = 128, 148
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/ (set to None
 # whenever the kernel changes after the counters were taken)
@@ -450,7 +452,7 @@ def run_ours(args):
         "timed": "CUDA events recorded by the library between the kernels of each layer's call, host queued ahead of the GPU; median of 72 calls",
         "alu": {"achieved": ALU_LANE_OPS_PER_UNIT * T * D / scan_s / 1e12, "peak": alu_peak / 1e12, "unit": "T fp32 lane-op/s",
                 "frac": ALU_LANE_OPS_PER_UNIT * T * D / scan_s / alu_peak,
-                "note": "this kernel is bound by fp32 instruction issue, not by HBM: 82 lane-ops and 8 bytes per token*channel (DESIGN.md)"},
+                "note": "this kernel is bound by fp32 instruction issue, not by HBM: 82 lane-ops and 8 bytes per token*channel"},
         "whole_prefill_call": {"us": call_s * 1e6, "achieved": pb / call_s / 1e9, "frac": pb / call_s / 1e9 / peak,
                                "summary_pass_us": split[0], "carry_scan_us": split[1], "output_pass_us": split[2],
                                "timed": "CUDA-graph replay of the 24 calls"},
