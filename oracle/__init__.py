@@ -58,6 +58,8 @@ def _bind(l):
     l.mdo_prefill.argtypes = [C.POINTER(_Layer), C.c_int, _c_int32_p] + [_c_double_p] * 10
     l.mdo_tree.restype = C.c_int
     l.mdo_tree.argtypes = [C.POINTER(_Layer), C.c_int, _c_int32_p] + [_c_double_p] * 10
+    l.mdo_tree_proj.restype = C.c_int
+    l.mdo_tree_proj.argtypes = [C.POINTER(_Layer), C.c_int, _c_double_p, _c_double_p, C.c_int, _c_int32_p] + [_c_double_p] * 10
     return l
 
 
@@ -160,6 +162,29 @@ def tree(layer: Layer, parents, x, z, dt, B, Cm, conv0=None, h0=None, flags=None
     if rc != 0:
         raise ValueError("parent indices must point to earlier nodes (or be -1)")
     return out, conv_nodes, h_nodes
+
+
+def tree_proj(layer: Layer, W_x, W_dt, parents, x, z, conv0=None, h0=None, flags=None, _lib_override=None):
+    """Draft tree of one sequence where the step size, B and C of a node are the block's projections of its conv
+    output: s = W_x u, dt = W_dt s[:R], B = s[R:R+N], C = s[R+N:].  W_x: (R+2N, D); W_dt: (D, R).
+    Returns (out (M,D), conv_nodes (M,W-1,D), h_nodes (M,D,N), dt (M,D), B (M,N), C (M,N))."""
+    L = _lib_override or lib()
+    Dn, N, W = layer.dims
+    W_dt = _f64(W_dt)
+    R = W_dt.shape[1]
+    W_dt = _f64(W_dt, (Dn, R)); W_x = _f64(W_x, (R + 2 * N, Dn))
+    par = np.ascontiguousarray(parents, dtype=np.int32)
+    M = par.shape[0]
+    x = _f64(x, (M, Dn)); z = _f64(z, (M, Dn))
+    conv0 = _f64(conv0, (W - 1, Dn)); h0 = _f64(h0, (Dn, N))
+    out = np.empty((M, Dn)); conv_nodes = np.empty((M, W - 1, Dn)); h_nodes = np.empty((M, Dn, N))
+    dt = np.empty((M, Dn)); B = np.empty((M, N)); Cm = np.empty((M, N))
+    cl = layer._c(flags)
+    rc = L.mdo_tree_proj(C.byref(cl), R, _p(W_x), _p(W_dt), M, par.ctypes.data_as(_c_int32_p), _p(x), _p(z), _p(conv0), _p(h0),
+                         _p(out), _p(conv_nodes), _p(h_nodes), _p(dt), _p(B), _p(Cm))
+    if rc != 0:
+        raise ValueError("parent indices must point to earlier nodes (or be -1)")
+    return out, conv_nodes, h_nodes, dt, B, Cm
 
 
 def layer_from_params(p, flags: int = DT_SOFTPLUS) -> Layer:

@@ -29,8 +29,11 @@
  * tiny inputs, scipy.signal.lfilter for the time-invariant case, numpy.convolve
  * and an impulse response for the conv, scalar identities for SiLU/softplus,
  * prefill hand-off, prefill == chain of steps, tree node == its root-to-node
- * path run as one short sequence, packed == each sequence alone.  The paper
- * prints no numeric value for this path, so no pin comes from a printed table.
+ * path run as one short sequence, packed == each sequence alone; for the tree
+ * with the block's projections: equality with the plain tree fed by numpy's
+ * matmul of the conv outputs, one-hot weights that turn both projections into
+ * gathers, zero weights (closed-form decay).  The paper prints no numeric value
+ * for this path, so no pin comes from a printed table.
  */
 #include <math.h>
 #include <stdint.h>
@@ -177,5 +180,83 @@ int mdo_tree(const mdo_layer *L, int M, const int32_t *parent,
         }
     }
     free(path);
+    return 0;
+}
+
+/*
+ * Tree drafting with the block's own selection projections.  The drafter is a
+ * Mamba model (paper Section 3.1, by citation), and in that block the step
+ * size, B and C of a token are not inputs: they are linear functions of the
+ * token's conv output u (all D channels of it),
+ *
+ *     s        = Wx * u                      Wx: (R + 2N, D)
+ *     dt[d]    = sum_{r<R} Wdt[d][r] * s[r]   Wdt: (D, R)     (dt_bias and softplus are applied as above)
+ *     B[n]     = s[R + n]
+ *     C[n]     = s[R + N + n]
+ *
+ * so a node is: conv step on every channel, the two projections, then the
+ * recurrence and the gate on every channel.  As in mdo_tree every node is
+ * rebuilt along its root-to-node path from the committed state (Section 4.1:
+ * a child needs only its parent's state).
+ *
+ * x, z: (M, D); out: (M, D); conv_nodes (M, W-1, D), h_nodes (M, D, N),
+ * dt_nodes (M, D), B_nodes (M, N), C_nodes (M, N) may each be NULL.
+ * Returns 0, or -1 if a parent index is not an earlier node.
+ */
+int mdo_tree_proj(const mdo_layer *L, int R, const double *Wx, const double *Wdt,
+                  int M, const int32_t *parent, const double *x, const double *z,
+                  const double *conv0, const double *h0,
+                  double *out, double *conv_nodes, double *h_nodes,
+                  double *dt_nodes, double *B_nodes, double *C_nodes)
+{
+    const int D = L->d_inner, N = L->d_state, W = L->d_conv;
+    for (int v = 0; v < M; ++v)
+        if (parent[v] >= v || parent[v] < -1) return -1;
+    mdo_layer conv_part = *L, scan_part = *L;
+    conv_part.flags = (L->flags & ~(uint32_t)MDO_PRECONV) | MDO_CONV_ONLY;
+    scan_part.flags = (L->flags & ~(uint32_t)MDO_CONV_ONLY) | MDO_PRECONV;
+    int *path = (int *)malloc(sizeof(int) * (size_t)(M > 0 ? M : 1));
+    double *win = (double *)malloc(sizeof(double) * (size_t)(W > 1 ? W - 1 : 1) * D);
+    double *h = (double *)malloc(sizeof(double) * (size_t)D * N);
+    double *u = (double *)malloc(sizeof(double) * (size_t)D);
+    double *dt = (double *)malloc(sizeof(double) * (size_t)D);
+    double *s = (double *)malloc(sizeof(double) * (size_t)(R + 2 * N));
+    for (int v = 0; v < M; ++v) {
+        int len = 0;
+        for (int a = v; a >= 0; a = parent[a]) path[len++] = a;
+        for (int d = 0; d < D; ++d) {
+            for (int k = 0; k < W - 1; ++k) win[(size_t)d * (W - 1) + k] = conv0 ? conv0[(size_t)k * D + d] : 0.0;
+            for (int n = 0; n < N; ++n) h[(size_t)d * N + n] = h0 ? h0[(size_t)d * N + n] : 0.0;
+        }
+        for (int j = len - 1; j >= 0; --j) {
+            const size_t a = (size_t)path[j];
+            for (int d = 0; d < D; ++d)
+                u[d] = channel_token(&conv_part, d, win + (size_t)d * (W - 1), NULL, x[a * D + d], 0.0, 0.0, NULL, NULL);
+            for (int r = 0; r < R + 2 * N; ++r) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) acc += Wx[(size_t)r * D + d] * u[d];
+                s[r] = acc;
+            }
+            for (int d = 0; d < D; ++d) {
+                double acc = 0.0;
+                for (int r = 0; r < R; ++r) acc += Wdt[(size_t)d * R + r] * s[r];
+                dt[d] = acc;
+            }
+            for (int d = 0; d < D; ++d)
+                out[(size_t)v * D + d] = channel_token(&scan_part, d, NULL, h + (size_t)d * N, u[d], z[a * D + d], dt[d], s + R, s + R + N);
+        }
+        for (int d = 0; d < D; ++d) {
+            if (conv_nodes)
+                for (int k = 0; k < W - 1; ++k) conv_nodes[((size_t)v * (W - 1) + k) * D + d] = win[(size_t)d * (W - 1) + k];
+            if (h_nodes)
+                for (int n = 0; n < N; ++n) h_nodes[((size_t)v * D + d) * N + n] = h[(size_t)d * N + n];
+            if (dt_nodes) dt_nodes[(size_t)v * D + d] = dt[d];
+        }
+        for (int n = 0; n < N; ++n) {
+            if (B_nodes) B_nodes[(size_t)v * N + n] = s[R + n];
+            if (C_nodes) C_nodes[(size_t)v * N + n] = s[R + N + n];
+        }
+    }
+    free(path); free(win); free(h); free(u); free(dt); free(s);
     return 0;
 }

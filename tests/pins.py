@@ -333,8 +333,78 @@ def pin_varlen(L=None):
     _close(cf[0, :1], ci[0, 2:], rtol=0, atol=0, what="2-token sequence shifts the window by two")
 
 
+def _proj_problem(i, Dn=6, N=3, R=2, M=9):
+    """Random tree problem for the projection pins; dense weights, every node with its own inputs."""
+    lay, x, z, _, _, _ = _random_problem(i, Dn=Dn, N=N, T=M)
+    g = _rng(100 + i)
+    Wx = g.normal(size=(R + 2 * N, Dn)); Wdt = g.normal(size=(Dn, R))
+    parents = np.array([-1, 0, 0, 1, 1, 2, 3, 3, 6][:M])
+    W = lay.dims[2]
+    c0 = g.normal(size=(W - 1, Dn)); h0 = g.normal(size=(Dn, N))
+    return lay, Wx, Wdt, parents, x, z, c0, h0
+
+
+def pin_proj_library_matmul(L=None):
+    """The projection tree == the plain tree fed with step size, B and C computed by numpy's matmul from the conv
+    outputs (conv outputs from the conv-only tree, itself pinned by the conv pins)."""
+    lay, Wx, Wdt, parents, x, z, c0, h0 = _proj_problem(20)
+    Dn, N, W = lay.dims
+    R = Wdt.shape[1]
+    out, cn, hn, dt, B, Cm = oracle.tree_proj(lay, Wx, Wdt, parents, x, z, conv0=c0, h0=h0, _lib_override=L)
+    zero = np.zeros_like(x); zbc = np.zeros((len(parents), N))
+    u, cu_nodes, _ = oracle.tree(lay, parents, x, zero, zero, zbc, zbc, conv0=c0, h0=h0, flags=lay.flags | oracle.CONV_ONLY, _lib_override=L)
+    s = np.matmul(u, Wx.T)
+    dt_ref = np.matmul(s[:, :R], Wdt.T)
+    _close(dt, dt_ref, what="dt = W_dt (W_x u)[:R]")
+    _close(B, s[:, R:R + N], what="B rows of W_x u")
+    _close(Cm, s[:, R + N:], what="C rows of W_x u")
+    o2, _, h2 = oracle.tree(lay, parents, u, z, dt_ref, s[:, R:R + N], s[:, R + N:], conv0=c0, h0=h0, flags=lay.flags | oracle.PRECONV, _lib_override=L)
+    _close(out, o2, what="projection tree: out")
+    _close(hn, h2, what="projection tree: state")
+    _close(cn, cu_nodes, rtol=0, atol=0, what="projection tree: conv window")
+
+
+def pin_proj_selectors(L=None):
+    """One-hot weights turn the projections into gathers: B[n] = u[n], C[n] = u[N+n], dt[d] = u[(d + 1) % R']."""
+    lay, _, _, parents, x, z, c0, h0 = _proj_problem(21, Dn=8, N=3, R=4)
+    Dn, N, W = lay.dims
+    R = 4
+    Wx = np.zeros((R + 2 * N, Dn)); Wdt = np.zeros((Dn, R))
+    for r in range(R): Wx[r, 7 - r] = 1.0                  # s[r] = u[7 - r]
+    for n in range(N): Wx[R + n, n] = 1.0; Wx[R + N + n, N + n] = 1.0
+    for d in range(Dn): Wdt[d, (d + 1) % R] = 1.0          # dt[d] = s[(d+1) % R] = u[7 - (d+1) % R]
+    out, _, hn, dt, B, Cm = oracle.tree_proj(lay, Wx, Wdt, parents, x, z, conv0=c0, h0=h0, _lib_override=L)
+    zero = np.zeros_like(x); zbc = np.zeros((len(parents), N))
+    u, _, _ = oracle.tree(lay, parents, x, zero, zero, zbc, zbc, conv0=c0, h0=h0, flags=lay.flags | oracle.CONV_ONLY, _lib_override=L)
+    _close(B, u[:, :N], rtol=0, atol=0, what="B gathers u[0:N]")
+    _close(Cm, u[:, N:2 * N], rtol=0, atol=0, what="C gathers u[N:2N]")
+    dsel = np.stack([u[:, 7 - (d + 1) % R] for d in range(Dn)], axis=1)
+    _close(dt, dsel, rtol=0, atol=0, what="dt gathers through both projections")
+    o2, _, h2 = oracle.tree(lay, parents, u, z, dsel, u[:, :N], u[:, N:2 * N], conv0=c0, h0=h0, flags=lay.flags | oracle.PRECONV, _lib_override=L)
+    _close(out, o2, rtol=0, atol=0, what="selector tree: out")
+    _close(hn, h2, rtol=0, atol=0, what="selector tree: state")
+
+
+def pin_proj_zero_weights(L=None):
+    """W_x = 0: dt = 0, B = C = 0, so out = D u SiLU(z) and the state only decays by exp(softplus(dt_bias) A) per step."""
+    lay, Wx, Wdt, parents, x, z, c0, h0 = _proj_problem(22)
+    Dn, N, W = lay.dims
+    out, _, hn, dt, B, Cm = oracle.tree_proj(lay, 0.0 * Wx, Wdt, parents, x, z, conv0=c0, h0=h0, _lib_override=L)
+    zero = np.zeros_like(x); zbc = np.zeros((len(parents), N))
+    u, _, _ = oracle.tree(lay, parents, x, zero, zero, zbc, zbc, conv0=c0, h0=h0, flags=lay.flags | oracle.CONV_ONLY, _lib_override=L)
+    _close(dt, zero, rtol=0, atol=0, what="zero W_x: dt"); _close(B, zbc, rtol=0, atol=0, what="zero W_x: B")
+    silu = np.vectorize(lambda v: v / (1.0 + math.exp(-v)))
+    _close(out, lay.D[None, :] * u * silu(z), what="zero W_x: out")
+    delta = np.array([math.log1p(math.exp(b)) for b in lay.dt_bias])
+    depth = np.zeros(len(parents), dtype=int)
+    for v in range(1, len(parents)): depth[v] = depth[parents[v]] + 1
+    for v in range(len(parents)):
+        _close(hn[v], np.exp(delta[:, None] * lay.A * (depth[v] + 1)) * h0, what=f"zero W_x: state of node {v}")
+
+
 ALL_PINS = [
     pin_scalar_functions, pin_geometric_series, pin_cumulative_sum, pin_frozen_state, pin_brute_force,
     pin_iir_filter, pin_softplus_and_bias_in_path, pin_conv_impulse, pin_conv_numpy,
     pin_conv_feeds_recurrence, pin_prefill_handoff, pin_prefill_equals_chain, pin_tree_paths, pin_varlen,
+    pin_proj_library_matmul, pin_proj_selectors, pin_proj_zero_weights,
 ]

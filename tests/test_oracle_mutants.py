@@ -31,6 +31,14 @@ MUTANTS = {
     "tree_ignores_committed_state": ("h[n] = h0 ? h0[(size_t)d * N + n] : 0.0;", "h[n] = 0.0;"),
     "gate_missing": ("return y * mdo_silu(z);", "return y;"),
     "state_transposed_A": ("exp(delta * L->A[(size_t)d * N + n])", "exp(delta * L->A[(size_t)n * L->d_inner + d < (size_t)L->d_inner * N ? (size_t)n * L->d_inner + d : 0])"),
+    "proj_from_raw_input": ("acc += Wx[(size_t)r * D + d] * u[d];", "acc += Wx[(size_t)r * D + d] * x[a * D + d];"),
+    "proj_Wx_transposed": ("acc += Wx[(size_t)r * D + d] * u[d];", "acc += Wx[(size_t)d * (R + 2 * N) + r] * u[d];"),
+    "proj_Wdt_transposed": ("acc += Wdt[(size_t)d * R + r] * s[r];", "acc += Wdt[(size_t)r * D + d] * s[r];"),
+    "proj_B_C_swapped": ("dt[d], s + R, s + R + N);", "dt[d], s + R + N, s + R);"),
+    "proj_dt_reads_B_rows": ("for (int r = 0; r < R; ++r) acc += Wdt[(size_t)d * R + r] * s[r];", "for (int r = 0; r < R; ++r) acc += Wdt[(size_t)d * R + r] * s[r + 1];"),
+    "proj_sum_drops_last_channel": ("for (int d = 0; d < D; ++d) acc += Wx[(size_t)r * D + d] * u[d];", "for (int d = 0; d + 1 < D; ++d) acc += Wx[(size_t)r * D + d] * u[d];"),
+    "proj_ignores_committed_state": ("h[(size_t)d * N + n] = h0 ? h0[(size_t)d * N + n] : 0.0;", "h[(size_t)d * N + n] = 0.0;"),
+    "proj_ignores_committed_window": ("win[(size_t)d * (W - 1) + k] = conv0 ? conv0[(size_t)k * D + d] : 0.0;", "win[(size_t)d * (W - 1) + k] = 0.0;"),
     "delta_softplus_skipped": ("(L->flags & MDO_DT_SOFTPLUS) ? mdo_softplus(v) : v;", "v;"),
 }
 
