@@ -15,6 +15,7 @@ from .configs import CONFIGS, Config, get_config
 from .draw import (
     LayerParams,
     layer_params,
+    select_proj,
     prefill_inputs,
     node_inputs,
     seq_lengths,

@@ -29,7 +29,7 @@ DT_PRE_LO = np.float32(-2.3125)
 DT_PRE_HI = np.float32(2.3125)
 
 _TENSOR_ID = {"x": 0, "z": 1, "dt": 2, "B": 3, "C": 4, "conv_w": 5, "conv_b": 6,
-              "lens": 7, "tree": 8, "accept": 9, "h0": 10, "conv0": 11}
+              "lens": 7, "tree": 8, "accept": 9, "h0": 10, "conv0": 11, "W_x": 12, "W_dt": 13}
 
 
 def rng_for(seed: int, cid: int, layer: int, rnd: int, tensor: str, phase: int = 0) -> np.random.Generator:
@@ -89,6 +89,17 @@ def layer_params(cfg: Config, layer: int, seed: Optional[int] = None, *,
         conv_b = (0.25 * rng_for(seed, cfg.cid, layer, 0, "conv_b").standard_normal(Dn, dtype=np.float32)).astype(np.float32)
     dt_bias = np.full(Dn, DT_BIAS, dtype=np.float32)
     return LayerParams(np.ascontiguousarray(A), Dskip, np.ascontiguousarray(conv_w), conv_b, dt_bias)
+
+
+def select_proj(cfg: Config, layer: int, dt_rank: int, seed: Optional[int] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Random weights of a block's two selection projections, in the activation dtype's values:
+    W_x (dt_rank + 2 N, D) ~ N(0, 1.6^2 / D) and W_dt (D, dt_rank) ~ N(0, 0.5^2 / dt_rank), scaled so that the
+    projected B, C and step-size pre-activation land near the spreads the direct recipe draws (1, 1 and 0.5)."""
+    seed = cfg.seed if seed is None else seed
+    Dn, N = cfg.d_inner, cfg.d_state
+    W_x = rng_for(seed, cfg.cid, layer, 0, "W_x").standard_normal((dt_rank + 2 * N, Dn), dtype=np.float32) * np.float32(1.6 / np.sqrt(Dn))
+    W_dt = rng_for(seed, cfg.cid, layer, 0, "W_dt").standard_normal((Dn, dt_rank), dtype=np.float32) * np.float32(0.5 / np.sqrt(dt_rank))
+    return round_to_act(W_x, cfg.act), round_to_act(W_dt, cfg.act)
 
 
 # ---------------------------------------------------------------- activations

@@ -212,6 +212,46 @@ int mdraft_tree_step(const mdraft_layer *layer, const mdraft_cache *cache, int32
                      int32_t *dev_status, void *stream);
 
 /*
+ * Draft-tree step with the block's own selection projections: like
+ * mdraft_tree_step for ONE level, but the step size, B and C of a node are not
+ * inputs; the call forms them from the node's conv output u (all d_inner
+ * channels) the way the drafter's Mamba block does (paper Section 3.1: the
+ * drafter is a Mamba model; Section 4.1: generation i is one batch of the
+ * level's nodes, each from its parent's state):
+ *
+ *     s     = W_x u                       W_x : (dt_rank + 2*d_state) x d_inner, row-major
+ *     dt[d] = sum_{r<dt_rank} W_dt[d][r] * s[r]     W_dt: d_inner x dt_rank, row-major
+ *     B[n]  = s[dt_rank + n],   C[n] = s[dt_rank + d_state + n]
+ *
+ * then dt_bias / softplus, the recurrence, the skip term and the gate exactly
+ * as in mdraft_tree_step.  u, s and dt are kept in fp32 from the conv to the
+ * recurrence (nothing is rounded to the activation dtype in between).  One
+ * launch per call; the blocks of a node exchange their shares of s through
+ * cluster shared memory, so no workspace is needed.
+ *
+ *   proj->W_x, proj->W_dt : device, activation dtype of the layer, 16-byte aligned, dense (no padding)
+ *   proj->dt_rank         : multiple of 8, 8..256
+ *   x, z, out             : device, n_nodes rows of d_inner activations (strides ldx, ldz, ldo in elements)
+ *   parent_slot, node_slot: device, n_nodes int32 each; same meaning and hazards as mdraft_tree_step
+ * layer->flags: MDRAFT_DT_SOFTPLUS and MDRAFT_A_POWERS are honoured; MDRAFT_PRECONV and
+ * MDRAFT_CONV_ONLY make no sense here (MDRAFT_ERR_INVALID_ARG).  d_inner above 4096 is
+ * MDRAFT_ERR_UNSUPPORTED (the blocks of a node must fit one cluster): use the split mode there.
+ * Device-side faults are reported through dev_status as in mdraft_tree_step.
+ */
+typedef struct mdraft_select_proj {
+    const void *W_x;
+    const void *W_dt;
+    int32_t dt_rank;
+    int32_t reserved;   /* 0 */
+} mdraft_select_proj;
+
+int mdraft_tree_step_proj(const mdraft_layer *layer, const mdraft_cache *cache, int32_t layer_index,
+                          const mdraft_select_proj *proj,
+                          const void *x, int64_t ldx, const void *z, int64_t ldz, void *out, int64_t ldo,
+                          int32_t n_nodes, const int32_t *parent_slot, const int32_t *node_slot,
+                          int32_t *dev_status, void *stream);
+
+/*
  * Accepted-path commit: for j in [0, n_commit) and every layer of the cache,
  * slot dst_slot[j] <- slot src_slot[j] (SSM state and conv window), bit for
  * bit.  After verification the drafter continues from the state of the last

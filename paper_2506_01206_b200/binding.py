@@ -25,7 +25,7 @@ MDRAFT_DEV_BAD_SLOT, MDRAFT_DEV_BAD_SEQLENS, MDRAFT_DEV_WAIT_EXPIRED = 1, 2, 4
 
 EXPORTS = (
     "mdraft_prefill_workspace_bytes", "mdraft_conv_scan_prefill", "mdraft_conv_scan_prefill_noalloc", "mdraft_tree_step",
-    "mdraft_state_commit", "mdraft_classify_A", "mdraft_status_string", "mdraft_version",
+    "mdraft_tree_step_proj", "mdraft_state_commit", "mdraft_classify_A", "mdraft_status_string", "mdraft_version",
     "mdraft_ucb_reward", "mdraft_ucb_select", "mdraft_ucb_update",
 )
 
@@ -52,6 +52,10 @@ class _Cache(C.Structure):
 class _PrefillOpts(C.Structure):
     _fields_ = [("chunk_len", C.c_int32), ("block_channels", C.c_int32), ("reserved", C.c_int32 * 2),
                 ("event_after_chunk_state", C.c_void_p), ("event_after_carry_scan", C.c_void_p)]
+
+
+class _SelectProj(C.Structure):
+    _fields_ = [("W_x", C.c_void_p), ("W_dt", C.c_void_p), ("dt_rank", C.c_int32), ("reserved", C.c_int32)]
 
 
 class _Ucb(C.Structure):
@@ -91,6 +95,9 @@ def load_library(path: Optional[str] = None):
     lib.mdraft_tree_step.argtypes = [C.POINTER(_Layer), C.POINTER(_Cache), i32,
                                      vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
                                      i32, vp, vp, i32, C.POINTER(i32), vp, vp]
+    lib.mdraft_tree_step_proj.restype = C.c_int
+    lib.mdraft_tree_step_proj.argtypes = [C.POINTER(_Layer), C.POINTER(_Cache), i32, C.POINTER(_SelectProj),
+                                          vp, i64, vp, i64, vp, i64, i32, vp, vp, vp, vp]
     lib.mdraft_state_commit.restype = C.c_int
     lib.mdraft_state_commit.argtypes = [C.POINTER(_Cache), i32, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.mdraft_classify_A.restype = C.c_int
@@ -299,6 +306,32 @@ def mdraft_tree_step(layer: Layer, cache: StateCache, layer_index: int, x, z, dt
                               M, _ptr(parent_slot), _ptr(node_slot), n_levels, lo, _ptr(dev_status), _stream_ptr(stream))
     if rc != 0:
         raise MdraftError(rc, "mdraft_tree_step")
+
+
+def mdraft_tree_step_proj(layer: Layer, cache: StateCache, layer_index: int, W_x: torch.Tensor, W_dt: torch.Tensor,
+                          x, z, out, parent_slot: torch.Tensor, node_slot: torch.Tensor,
+                          dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None) -> None:
+    """One tree level where dt, B and C come from the block's projections of the conv output.
+    W_x: (dt_rank + 2 N, D) and W_dt: (D, dt_rank), contiguous, in the layer's activation dtype."""
+    lib = load_library()
+    cl = layer.c(flags)
+    cc = cache.c()
+    px, ldx = _mat(x, "x"); pz, ldz = _mat(z, "z"); po, ldo = _mat(out, "out")
+    M = int(x.shape[0])
+    if parent_slot.dtype != torch.int32 or node_slot.dtype != torch.int32:
+        raise TypeError("slot index arrays must be int32")
+    if parent_slot.numel() != M or node_slot.numel() != M:
+        raise ValueError("one parent slot and one node slot per node")
+    if W_x.dtype != x.dtype or W_dt.dtype != x.dtype or not W_x.is_contiguous() or not W_dt.is_contiguous():
+        raise TypeError("W_x and W_dt must be contiguous and of the activation dtype")
+    R = int(W_dt.shape[1])
+    if tuple(W_dt.shape) != (layer.d_inner, R) or tuple(W_x.shape) != (R + 2 * layer.d_state, layer.d_inner):
+        raise ValueError("W_x must be (dt_rank + 2 d_state, d_inner) and W_dt (d_inner, dt_rank)")
+    pr = _SelectProj(W_x.data_ptr(), W_dt.data_ptr(), R, 0)
+    rc = lib.mdraft_tree_step_proj(C.byref(cl), C.byref(cc), int(layer_index), C.byref(pr), px, ldx, pz, ldz, po, ldo,
+                                   M, _ptr(parent_slot), _ptr(node_slot), _ptr(dev_status), _stream_ptr(stream))
+    if rc != 0:
+        raise MdraftError(rc, "mdraft_tree_step_proj")
 
 
 def mdraft_state_commit(cache: StateCache, src_slot: torch.Tensor, dst_slot: torch.Tensor,

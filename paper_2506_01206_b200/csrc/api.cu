@@ -7,6 +7,7 @@
 #include "commit.cuh"
 #include "common.cuh"
 #include "prefill.cuh"
+#include "tree_proj.cuh"
 #include "tree_step.cuh"
 
 using namespace mdraft;
@@ -294,6 +295,36 @@ int mdraft_tree_step(const mdraft_layer* layer, const mdraft_cache* cache, int32
         a.lvl_end = level_offsets ? level_offsets[l + 1] : n_nodes;
         if (launch_tree_step(a, act, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MDRAFT_ERR_CUDA;
     }
+    return MDRAFT_OK;
+}
+
+int mdraft_tree_step_proj(const mdraft_layer* layer, const mdraft_cache* cache, int32_t layer_index,
+                          const mdraft_select_proj* proj, const void* x, int64_t ldx, const void* z, int64_t ldz, void* out,
+                          int64_t ldo, int32_t n_nodes, const int32_t* parent_slot, const int32_t* node_slot,
+                          int32_t* dev_status, void* stream) {
+    int rc = check_layer(layer);
+    if (rc) return rc;
+    if ((rc = check_cache(cache, layer->d_inner, layer->act, layer_index))) return rc;
+    if (layer->flags & (MDRAFT_PRECONV | MDRAFT_CONV_ONLY)) return MDRAFT_ERR_INVALID_ARG;
+    if (!proj || !proj->W_x || !proj->W_dt || n_nodes < 0) return MDRAFT_ERR_INVALID_ARG;
+    if (!aligned16(proj->W_x) || !aligned16(proj->W_dt)) return MDRAFT_ERR_MISALIGNED;
+    if (proj->dt_rank < 8 || proj->dt_rank > kProjMaxRank || (proj->dt_rank % 8) != 0) return MDRAFT_ERR_UNSUPPORTED;
+    if (tree_proj_block_channels(layer->d_inner) == 0) return MDRAFT_ERR_UNSUPPORTED;
+    if (n_nodes == 0) return MDRAFT_OK;
+    if (!parent_slot || !node_slot) return MDRAFT_ERR_INVALID_ARG;
+    const int D = layer->d_inner, act = layer->act;
+    if ((rc = check_matrix(x, ldx, D, act, true))) return rc;
+    if ((rc = check_matrix(z, ldz, D, act, true))) return rc;
+    if ((rc = check_matrix(out, ldo, D, act, true))) return rc;
+
+    TreeProjArgs a;
+    a.L = layer_dev(layer);
+    a.pool = pool_dev(cache, act, layer_index);
+    a.x = x; a.z = z; a.out = out;
+    a.ldx = ldx; a.ldz = ldz; a.ldo = ldo;
+    a.W_x = proj->W_x; a.W_dt = proj->W_dt; a.dt_rank = proj->dt_rank;
+    a.parent_slot = parent_slot; a.node_slot = node_slot; a.n_nodes = n_nodes; a.dev_status = dev_status;
+    if (launch_tree_proj(a, act, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MDRAFT_ERR_CUDA;
     return MDRAFT_OK;
 }
 

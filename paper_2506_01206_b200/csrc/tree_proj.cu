@@ -1,0 +1,355 @@
+// Draft-tree step of a whole Mamba block core: conv step, the block's two selection projections, recurrence, gate.
+//
+// In the drafter's block the step size, B and C of a token are linear functions of the conv output of ALL channels
+// (s = W_x u; dt = W_dt s[0:R]; B = s[R:R+N]; C = s[R+N:R+2N]), so between the conv step and the recurrence sits a
+// reduction over the channel axis.  Here the blocks of one node form a thread-block cluster along the channel axis:
+// every block convolves its channels, multiplies them into its share of s (a partial sum per row of W_x), the
+// cluster meets at its hardware barrier, every block adds the partial sums of all blocks out of their shared memory
+// (distributed shared memory, fixed order, so all blocks hold the same bits), forms the step size of its own channels
+// from its rows of W_dt and advances the recurrence.  One launch per tree level replaces the conv step, two
+// matrix products, three slicing copies and the recurrence step of the split mode; nothing goes through global
+// memory in between.
+//
+// The parent's state slice, window rows and the node's x / z rows arrive by bulk asynchronous copies counted on two
+// mbarriers (window and x first, state and z later, so the projections overlap the 16-32 KB state fetch); the child's
+// state, window and output leave by bulk stores.  All waits on the mbarriers are bounded.  The cluster barrier is
+// executed unconditionally by every thread of every block of the cluster (a block that gave up on its copies still
+// takes part), so no block can wait for one that left.
+#include "common.cuh"
+#include "tree_proj.cuh"
+
+namespace mdraft {
+
+namespace {
+
+constexpr uint32_t kSpinLimit = 1u << 20;  // polls of an mbarrier before the block gives up
+constexpr int kMaxRows = kProjMaxRank + 2 * kN;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+// Bulk copies; addresses 16-byte aligned, sizes multiples of 16 bytes.  The destination and the mbarrier are this
+// block's own shared memory (a block's own addresses are valid in the cluster window).
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+                 "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(dst)), "r"(smem_u32(src)),
+                 "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
+    return n;
+}
+// The float that block `rank` of this cluster keeps at the place where this block keeps *local.
+__device__ __forceinline__ float peer_block_float(const float* local, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local)), "r"(rank));
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void swap4(float4& a, float4& b) { const float4 t = a; a = b; b = t; }
+__device__ __forceinline__ void xor_permute(float4 (&t)[4], int sw) {
+    if (sw & 1) { swap4(t[0], t[1]); swap4(t[2], t[3]); }
+    if (sw & 2) { swap4(t[0], t[2]); swap4(t[1], t[3]); }
+}
+
+// Four consecutive weights as floats.
+__device__ __forceinline__ float4 load_w4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load_w4(const __nv_bfloat16* p) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
+                       __uint_as_float(v.y & 0xffff0000u));
+}
+__device__ __forceinline__ float dot4(const float4& a, const float4& b, float acc) {
+    acc = fmaf(a.x, b.x, acc); acc = fmaf(a.y, b.y, acc); acc = fmaf(a.z, b.z, acc); acc = fmaf(a.w, b.w, acc);
+    return acc;
+}
+
+template <typename AT, int CB, bool kPow>
+__global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
+    constexpr int NW = CB / 32;    // warps
+    constexpr int NP = CB / 128;   // a lane owns 4 consecutive channels in each of NP 128-channel spans
+    __shared__ __align__(128) float4 s_h[CB * (kN / 4)];  // state slice [channel][quad]
+    __shared__ __align__(16) AT s_conv[kW - 1][CB];
+    __shared__ __align__(16) AT s_x[CB];                  // the node's x row; receives the out row afterwards
+    __shared__ __align__(16) AT s_z[CB];
+    __shared__ __align__(16) float s_u[CB];               // conv outputs of this block's channels
+    __shared__ __align__(16) float s_part[kMaxRows];      // this block's share of s = W_x u
+    __shared__ __align__(16) float s_s[kMaxRows];         // s, summed over the cluster
+    __shared__ __align__(8) uint64_t bar_a, bar_b;
+
+    const int D = p.L.d_inner, R = p.dt_rank, rows = R + 2 * kN;
+    const int node = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int d0 = blockIdx.y * CB;
+    const int cols = min(CB, D - d0);
+    const int d = d0 + tid;
+    const bool live = tid < cols;
+    const int pslot = __ldg(p.parent_slot + node);
+    const int nslot = __ldg(p.node_slot + node);
+    // The slots are the node's, so every block of the cluster takes the same way out here, before any barrier.
+    if (pslot < -1 || pslot >= p.pool.n_slots || nslot < 0 || nslot >= p.pool.n_slots) {
+        if (tid == 0 && blockIdx.y == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+        return;
+    }
+    const uint32_t flags = p.L.flags;
+    const bool have_parent = pslot >= 0;
+    const uint32_t row_bytes = (uint32_t)cols * sizeof(AT), h_bytes = (uint32_t)cols * kN * 4u;
+    float* h_parent = p.pool.ssm + (size_t)pslot * p.pool.ssm_slot_stride + (size_t)d0 * kN;
+    float* h_child = p.pool.ssm + (size_t)nslot * p.pool.ssm_slot_stride + (size_t)d0 * kN;
+    AT* conv_parent = static_cast<AT*>(p.pool.conv) + (size_t)pslot * p.pool.conv_slot_stride + d0;
+    AT* conv_child = static_cast<AT*>(p.pool.conv) + (size_t)nslot * p.pool.conv_slot_stride + d0;
+
+    if (tid == 0) {
+        mbar_init(&bar_a, 1);
+        mbar_init(&bar_b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(&bar_a, row_bytes + (have_parent ? (kW - 1) * row_bytes : 0u));
+        bulk_load(s_x, static_cast<const AT*>(p.x) + (size_t)node * p.ldx + d0, row_bytes, &bar_a);
+        if (have_parent)
+            for (int j = 0; j < kW - 1; ++j) bulk_load(s_conv[j], conv_parent + (size_t)j * D, row_bytes, &bar_a);
+        mbar_expect_tx(&bar_b, row_bytes + (have_parent ? h_bytes : 0u));
+        if (have_parent) bulk_load(s_h, h_parent, h_bytes, &bar_b);
+        bulk_load(s_z, static_cast<const AT*>(p.z) + (size_t)node * p.ldz + d0, row_bytes, &bar_b);
+    }
+
+    // Layer constants travel by ordinary loads while the copies are in flight.
+    float a2[kPow ? 1 : kN];
+    float4 wv = make_float4(0.f, 0.f, 0.f, 0.f);
+    float cb = 0.f, dtb = 0.f, dsk = 0.f;
+    if (live) {
+        wv = __ldg(reinterpret_cast<const float4*>(p.L.conv_w + (size_t)d * kW));
+        cb = p.L.conv_b ? __ldg(p.L.conv_b + d) : 0.f;
+        if constexpr (kPow) {
+            a2[0] = __ldg(p.L.A + (size_t)d * kN) * kLog2e;
+        } else {
+#pragma unroll
+            for (int q = 0; q < kN / 4; ++q) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(p.L.A + (size_t)d * kN) + q);
+                a2[4 * q] = a.x * kLog2e; a2[4 * q + 1] = a.y * kLog2e; a2[4 * q + 2] = a.z * kLog2e; a2[4 * q + 3] = a.w * kLog2e;
+            }
+        }
+        dtb = p.L.dt_bias ? __ldg(p.L.dt_bias + d) : 0.f;
+        dsk = p.L.D ? __ldg(p.L.D + d) : 0.f;
+    }
+    __syncthreads();  // the mbarriers are initialised for everyone
+    bool bad = __syncthreads_or(!mbar_wait_bounded(&bar_a, 0u));
+
+    // ---- conv window: (w0, w1, w2, x) -> (w1, w2, x)
+    float u = 0.f;
+    if (live && !bad) {
+        const float xv = Act<AT>::to_f32(s_x[tid]);
+        float win[kW - 1] = {0.f, 0.f, 0.f};
+        if (have_parent) {
+#pragma unroll
+            for (int j = 0; j < kW - 1; ++j) win[j] = Act<AT>::to_f32(s_conv[j][tid]);
+        }
+        float acc = fmaf(wv.x, win[0], cb);
+        acc = fmaf(wv.y, win[1], acc);
+        acc = fmaf(wv.z, win[2], acc);
+        acc = fmaf(wv.w, xv, acc);
+        u = silu(acc);
+        s_conv[0][tid] = Act<AT>::from_f32(win[1]);
+        s_conv[1][tid] = Act<AT>::from_f32(win[2]);
+        s_conv[2][tid] = Act<AT>::from_f32(xv);
+    }
+    s_u[tid] = u;
+    __syncthreads();
+
+    // ---- this block's share of s = W_x u: a warp takes every NW-th row, a lane 4 NP channels of it.
+    {
+        float4 uu[NP];
+        bool in[NP];
+#pragma unroll
+        for (int q = 0; q < NP; ++q) {
+            uu[q] = *reinterpret_cast<const float4*>(&s_u[q * 128 + 4 * lane]);
+            in[q] = q * 128 + 4 * lane < cols;  // cols is a multiple of 8: a group of four is all in or all out
+        }
+        const AT* wx = static_cast<const AT*>(p.W_x) + d0 + 4 * lane;
+        constexpr int kBatch = 4;  // rows in flight per warp
+        for (int r0 = warp; r0 < rows; r0 += kBatch * NW) {
+            float acc[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const int r = r0 + j * NW;
+                acc[j] = 0.f;
+                if (r < rows) {
+#pragma unroll
+                    for (int q = 0; q < NP; ++q)
+                        if (in[q]) acc[j] = dot4(load_w4(wx + (size_t)r * D + q * 128), uu[q], acc[j]);
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j)
+                    if (r0 + j * NW < rows) s_part[r0 + j * NW] = acc[j];
+            }
+        }
+    }
+    // Every block's share is complete and visible to the cluster after this barrier.
+    cluster_arrive();
+    cluster_wait();
+    {
+        const uint32_t nblk = cluster_size();
+        for (int r = tid; r < rows; r += CB) {
+            float sum = 0.f;
+            for (uint32_t c = 0; c < nblk; ++c) sum += peer_block_float(&s_part[r], c);
+            s_s[r] = sum;
+        }
+    }
+    cluster_arrive();  // this block no longer reads its neighbours; the matching wait is the last thing it does
+    __syncthreads();
+
+    // ---- step size of this thread's channel: dt = W_dt[d][:] . s[0:R]  (R is a multiple of 8)
+    float dtv = 0.f;
+    if (live) {
+        const AT* wr = static_cast<const AT*>(p.W_dt) + (size_t)d * R;
+        float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll 2
+        for (int r = 0; r < R; r += 8) {
+            const float4 w0 = load_w4(wr + r), w1 = load_w4(wr + r + 4);
+            acc0 = dot4(w0, *reinterpret_cast<const float4*>(&s_s[r]), acc0);
+            acc1 = dot4(w1, *reinterpret_cast<const float4*>(&s_s[r + 4]), acc1);
+        }
+        dtv = acc0 + acc1;
+    }
+
+    bad = __syncthreads_or(bad || !mbar_wait_bounded(&bar_b, 0u));
+
+    if (live && !bad) {
+        // ---- one step of the recurrence.  The quads of a channel are visited in an order that differs between
+        // neighbouring threads, which keeps the 128-bit shared-memory accesses free of bank conflicts.
+        const int sw = (tid >> 1) & 3;
+        float4 hq[kN / 4];
+#pragma unroll
+        for (int i = 0; i < kN / 4; ++i) hq[i] = have_parent ? s_h[tid * (kN / 4) + (i ^ sw)] : make_float4(0.f, 0.f, 0.f, 0.f);
+        xor_permute(hq, sw);
+        const float zv = Act<AT>::to_f32(s_z[tid]);
+        const float v = dtv + dtb;
+        const float delta = (flags & MDRAFT_DT_SOFTPLUS) ? softplus(v) : v;
+        const float du = delta * u;
+        float P[kN];
+        if constexpr (kPow) {
+            const float r1 = ex2(delta * a2[0]);
+            const float r2 = r1 * r1, r4 = r2 * r2, r8 = r4 * r4;
+            P[0] = r1; P[1] = r2; P[2] = r2 * r1; P[3] = r4;
+            P[4] = r4 * r1; P[5] = r4 * r2; P[6] = r4 * P[2]; P[7] = r8;
+#pragma unroll
+            for (int n = 0; n < 8; ++n) P[8 + n] = r8 * P[n];
+        } else {
+#pragma unroll
+            for (int n = 0; n < kN; ++n) P[n] = ex2(delta * a2[n]);
+        }
+        float h[kN], Bv[kN], Cv[kN];
+#pragma unroll
+        for (int q = 0; q < kN / 4; ++q) {
+            h[4 * q] = hq[q].x; h[4 * q + 1] = hq[q].y; h[4 * q + 2] = hq[q].z; h[4 * q + 3] = hq[q].w;
+            const float4 b = *reinterpret_cast<const float4*>(&s_s[R + 4 * q]);
+            const float4 c = *reinterpret_cast<const float4*>(&s_s[R + kN + 4 * q]);
+            Bv[4 * q] = b.x; Bv[4 * q + 1] = b.y; Bv[4 * q + 2] = b.z; Bv[4 * q + 3] = b.w;
+            Cv[4 * q] = c.x; Cv[4 * q + 1] = c.y; Cv[4 * q + 2] = c.z; Cv[4 * q + 3] = c.w;
+        }
+        float y0 = 0.f, y1 = 0.f;
+#pragma unroll
+        for (int n = 0; n < kN; ++n) {
+            h[n] = fmaf(P[n], h[n], du * Bv[n]);
+            if (n & 1) y1 = fmaf(Cv[n], h[n], y1); else y0 = fmaf(Cv[n], h[n], y0);
+        }
+#pragma unroll
+        for (int q = 0; q < kN / 4; ++q) hq[q] = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
+        xor_permute(hq, sw);
+#pragma unroll
+        for (int i = 0; i < kN / 4; ++i) s_h[tid * (kN / 4) + (i ^ sw)] = hq[i];
+        s_x[tid] = Act<AT>::from_f32(fmaf(dsk, u, y0 + y1) * silu(zv));
+    }
+    // Shared-memory writes above must be visible to the copy engine before it reads them.
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    if (tid == 0) {
+        if (bad) {
+            // Nothing of this node is stored.  The copies target this block's shared memory: give them one more
+            // bounded chance to land before the block ends.
+            flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
+            mbar_wait_bounded(&bar_a, 0u);
+            mbar_wait_bounded(&bar_b, 0u);
+        } else {
+            bulk_store(h_child, s_h, h_bytes);
+            for (int j = 0; j < kW - 1; ++j) bulk_store(conv_child + (size_t)j * D, s_conv[j], row_bytes);
+            bulk_store(static_cast<AT*>(p.out) + (size_t)node * p.ldo + d0, s_x, row_bytes);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory stays valid until it has been read
+        }
+    }
+    __syncwarp();
+    cluster_wait();  // no block of the cluster leaves while a neighbour may still read its share of s
+}
+
+template <typename AT, int CB>
+cudaError_t launch_cb(const TreeProjArgs& p, int n_blocks, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.n_nodes, (unsigned)n_blocks, 1);
+    cfg.blockDim = dim3(CB, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 1;
+    at[0].val.clusterDim.y = (unsigned)n_blocks;  // the blocks of one node
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (p.L.flags & MDRAFT_A_POWERS) return cudaLaunchKernelEx(&cfg, tree_proj_kernel<AT, CB, true>, p);
+    return cudaLaunchKernelEx(&cfg, tree_proj_kernel<AT, CB, false>, p);
+}
+
+template <typename AT>
+cudaError_t launch_act(const TreeProjArgs& p, cudaStream_t st) {
+    const int cb = tree_proj_block_channels(p.L.d_inner);
+    const int n_blocks = (p.L.d_inner + cb - 1) / cb;
+    switch (cb) {
+        case 128: return launch_cb<AT, 128>(p, n_blocks, st);
+        case 256: return launch_cb<AT, 256>(p, n_blocks, st);
+        case 512: return launch_cb<AT, 512>(p, n_blocks, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+int tree_proj_block_channels(int d_inner) {
+    for (int cb = 128; cb <= 512; cb *= 2)
+        if ((d_inner + cb - 1) / cb <= kProjMaxCluster) return cb;
+    return 0;
+}
+
+cudaError_t launch_tree_proj(const TreeProjArgs& p, int act, cudaStream_t st) {
+    if (p.n_nodes <= 0) return cudaSuccess;
+    return act == MDRAFT_F32 ? launch_act<float>(p, st) : launch_act<__nv_bfloat16>(p, st);
+}
+
+}  // namespace mdraft
