@@ -80,6 +80,41 @@ __device__ __forceinline__ float4 load_w4(const __nv_bfloat16* p) {
     return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
                        __uint_as_float(v.y & 0xffff0000u));
 }
+// Eight consecutive weights, kept as loaded until they are used.
+template <typename AT> struct Raw8;
+template <> struct Raw8<float> {
+    float4 a, b;
+    __device__ __forceinline__ void load(const float* p) { a = load_w4(p); b = load_w4(p + 4); }
+    __device__ __forceinline__ float4 lo() const { return a; }
+    __device__ __forceinline__ float4 hi() const { return b; }
+};
+template <> struct Raw8<__nv_bfloat16> {
+    uint4 v;
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint4*>(p)); }
+    __device__ __forceinline__ float4 lo() const {
+        return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
+                           __uint_as_float(v.y & 0xffff0000u));
+    }
+    __device__ __forceinline__ float4 hi() const {
+        return make_float4(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u), __uint_as_float(v.w << 16),
+                           __uint_as_float(v.w & 0xffff0000u));
+    }
+};
+// Four consecutive weights as loaded (8 or 16 bytes).
+template <typename AT> struct Raw4;
+template <> struct Raw4<float> {
+    float4 v;
+    __device__ __forceinline__ void load(const float* p) { v = load_w4(p); }
+    __device__ __forceinline__ float4 get() const { return v; }
+};
+template <> struct Raw4<__nv_bfloat16> {
+    uint2 v;
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint2*>(p)); }
+    __device__ __forceinline__ float4 get() const {
+        return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
+                           __uint_as_float(v.y & 0xffff0000u));
+    }
+};
 __device__ __forceinline__ float dot4(const float4& a, const float4& b, float acc) {
     acc = fmaf(a.x, b.x, acc); acc = fmaf(a.y, b.y, acc); acc = fmaf(a.z, b.z, acc); acc = fmaf(a.w, b.w, acc);
     return acc;
@@ -152,6 +187,30 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
         dtb = p.L.dt_bias ? __ldg(p.L.dt_bias + d) : 0.f;
         dsk = p.L.D ? __ldg(p.L.D + d) : 0.f;
     }
+    // The weights depend on nothing that is still in flight: the first rows of this warp's share of W_x and the
+    // head of this channel's row of W_dt are requested now, ahead of the waits they would otherwise queue behind.
+    constexpr int kPreRows = NP == 4 ? (sizeof(AT) == 4 ? 3 : 5) : 10;  // rows of W_x held in registers per warp
+    constexpr int kPreDt = sizeof(AT) == 4 ? 3 : 6;  // groups of eight weights of W_dt held in registers per thread
+    const AT* wx = static_cast<const AT*>(p.W_x) + d0 + 4 * lane;
+    bool in[NP];
+#pragma unroll
+    for (int q = 0; q < NP; ++q) in[q] = q * 128 + 4 * lane < cols;  // cols is a multiple of 8: a group of four is all in or all out
+    Raw4<AT> wpre[kPreRows][NP];
+#pragma unroll
+    for (int j = 0; j < kPreRows; ++j) {
+        const int r = warp + j * NW;
+#pragma unroll
+        for (int q = 0; q < NP; ++q) {
+            wpre[j][q].load(wx);  // a valid address; replaced below when the row and the channels exist
+            if (r < rows && in[q]) wpre[j][q].load(wx + (size_t)r * D + q * 128);
+        }
+    }
+    const AT* wr = static_cast<const AT*>(p.W_dt) + (size_t)(live ? d : d0) * R;
+    Raw8<AT> dpre[kPreDt];
+#pragma unroll
+    for (int j = 0; j < kPreDt; ++j)
+        dpre[j].load(wr + (8 * j < R ? 8 * j : 0));
+
     __syncthreads();  // the mbarriers are initialised for everyone
     bool bad = __syncthreads_or(!mbar_wait_bounded(&bar_a, 0u));
 
@@ -179,35 +238,49 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
     // ---- this block's share of s = W_x u: a warp takes every NW-th row, a lane 4 NP channels of it.
     {
         float4 uu[NP];
-        bool in[NP];
 #pragma unroll
-        for (int q = 0; q < NP; ++q) {
-            uu[q] = *reinterpret_cast<const float4*>(&s_u[q * 128 + 4 * lane]);
-            in[q] = q * 128 + 4 * lane < cols;  // cols is a multiple of 8: a group of four is all in or all out
+        for (int q = 0; q < NP; ++q) uu[q] = *reinterpret_cast<const float4*>(&s_u[q * 128 + 4 * lane]);
+        float acc[kPreRows];
+#pragma unroll
+        for (int j = 0; j < kPreRows; ++j) {
+            acc[j] = 0.f;
+#pragma unroll
+            for (int q = 0; q < NP; ++q)
+                if (in[q]) acc[j] = dot4(wpre[j][q].get(), uu[q], acc[j]);
         }
-        const AT* wx = static_cast<const AT*>(p.W_x) + d0 + 4 * lane;
-        constexpr int kBatch = 4;  // rows in flight per warp
-        for (int r0 = warp; r0 < rows; r0 += kBatch * NW) {
-            float acc[kBatch];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int j = 0; j < kPreRows; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int j = 0; j < kPreRows; ++j)
+                if (warp + j * NW < rows) s_part[warp + j * NW] = acc[j];
+        }
+        // Rows beyond the prefetched ones (large dt_rank), four in flight per warp.
+        constexpr int kBatch = 4;
+        for (int r0 = warp + kPreRows * NW; r0 < rows; r0 += kBatch * NW) {
+            float a4[kBatch];
 #pragma unroll
             for (int j = 0; j < kBatch; ++j) {
                 const int r = r0 + j * NW;
-                acc[j] = 0.f;
+                a4[j] = 0.f;
                 if (r < rows) {
 #pragma unroll
                     for (int q = 0; q < NP; ++q)
-                        if (in[q]) acc[j] = dot4(load_w4(wx + (size_t)r * D + q * 128), uu[q], acc[j]);
+                        if (in[q]) a4[j] = dot4(load_w4(wx + (size_t)r * D + q * 128), uu[q], a4[j]);
                 }
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-                for (int j = 0; j < kBatch; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+                for (int j = 0; j < kBatch; ++j) a4[j] += __shfl_xor_sync(0xffffffffu, a4[j], o);
             }
             if (lane == 0) {
 #pragma unroll
                 for (int j = 0; j < kBatch; ++j)
-                    if (r0 + j * NW < rows) s_part[r0 + j * NW] = acc[j];
+                    if (r0 + j * NW < rows) s_part[r0 + j * NW] = a4[j];
             }
         }
     }
@@ -228,10 +301,16 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
     // ---- step size of this thread's channel: dt = W_dt[d][:] . s[0:R]  (R is a multiple of 8)
     float dtv = 0.f;
     if (live) {
-        const AT* wr = static_cast<const AT*>(p.W_dt) + (size_t)d * R;
         float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < kPreDt; ++j) {
+            if (8 * j < R) {
+                acc0 = dot4(dpre[j].lo(), *reinterpret_cast<const float4*>(&s_s[8 * j]), acc0);
+                acc1 = dot4(dpre[j].hi(), *reinterpret_cast<const float4*>(&s_s[8 * j + 4]), acc1);
+            }
+        }
 #pragma unroll 2
-        for (int r = 0; r < R; r += 8) {
+        for (int r = 8 * kPreDt; r < R; r += 8) {
             const float4 w0 = load_w4(wr + r), w1 = load_w4(wr + r + 4);
             acc0 = dot4(w0, *reinterpret_cast<const float4*>(&s_s[r]), acc0);
             acc1 = dot4(w1, *reinterpret_cast<const float4*>(&s_s[r + 4]), acc1);
