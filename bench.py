@@ -504,28 +504,31 @@ def run_ours(args):
     }
 
     # ---- context figure: drafting latency per round of a whole 130M-shaped block stack with real data dependence
-    # (split mode: conv step -> projections -> S6 step; torch matmuls on random weights for the projections, one CUDA
-    # graph per generation step), the quantity of the paper's Table 4.  Not part of `value`.
+    # (split mode: conv step -> torch matmuls for the projections -> S6 step; projection step: one launch that does
+    # all of it; random weights, one CUDA graph per generation step), the quantity of the paper's Table 4.  Not part
+    # of `value`.
     drafter = None
     if rank == 0 and world == 1:
         from paper_2506_01206_b200.drafter import ToyDrafter
-        td = ToyDrafter(max_nodes=64, seed=0, device=dev)
         drafter = {"unit": "ms per draft round (host launches and top-k between generation steps included)",
                    "paper_context": "6.62 (chain of 5) and 8.30 (tree (3,2,2,1,1)) on an RTX 4090, unit unstated, Mamba-130M drafter (paper Table 4)"}
-        for name, cfg_t in (("chain_5", (1, 1, 1, 1, 1)), ("tree_3_2_2_1_1", (3, 2, 2, 1, 1))):
-            for _ in range(3):
-                td.draft_round(11, cfg_t)
-            torch.cuda.synchronize()
-            ts = []
-            for _ in range(10):
-                t0 = time.perf_counter()
-                td.draft_round(11, cfg_t)
+        for mode, fused in (("split_mode", False), ("projection_step", True)):
+            td = ToyDrafter(max_nodes=64, seed=0, device=dev, fused=fused)
+            drafter[mode] = {}
+            for name, cfg_t in (("chain_5", (1, 1, 1, 1, 1)), ("tree_3_2_2_1_1", (3, 2, 2, 1, 1))):
+                for _ in range(3):
+                    td.draft_round(11, cfg_t)
                 torch.cuda.synchronize()
-                ts.append((time.perf_counter() - t0) * 1e3)
-            drafter[name] = statistics.median(ts)
-        if int(td.status.item()):
-            raise RuntimeError("device status bits set in the drafter leg")
-        del td
+                ts = []
+                for _ in range(10):
+                    t0 = time.perf_counter()
+                    td.draft_round(11, cfg_t)
+                    torch.cuda.synchronize()
+                    ts.append((time.perf_counter() - t0) * 1e3)
+                drafter[mode][name] = statistics.median(ts)
+            if int(td.status.item()):
+                raise RuntimeError("device status bits set in the drafter leg")
+            del td
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:

@@ -1,8 +1,10 @@
 """A Mamba drafter block stack around the library, with the data dependence a real drafter has.
 
 In a Mamba block the step size, B and C are projections of the conv output, so the fused conv+scan call cannot be
-fed by a real model; the library's split mode is for that: `MDRAFT_CONV_ONLY` (conv window + SiLU), the caller's
-projections, then `MDRAFT_PRECONV` (recurrence + gate).  This module is that caller, for drafting only: embedding,
+fed by a real model.  The library offers two ways: the split mode, `MDRAFT_CONV_ONLY` (conv window + SiLU), the
+caller's projections, then `MDRAFT_PRECONV` (recurrence + gate); or `mdraft_tree_step_proj`, which takes the two
+projection matrices and does conv step, projections, recurrence and gate in one launch (`fused=True` here).  This
+module is the caller, for drafting only: embedding,
 24 x [RMSNorm, in_proj, conv step, x_proj, dt_proj, S6 step, out_proj, residual], final norm, LM head, and
 tree-structured drafting by batch generation (paper Section 4.1): generation i is one batch of all nodes of level
 i, each node forks its parent's conv / SSM state by slot index, and the children of a node are its N_i most
@@ -24,7 +26,7 @@ from . import binding as mb
 
 class ToyDrafter:
     def __init__(self, n_layers: int = 24, d_model: int = 768, d_inner: int = 1536, dt_rank: int = 48, vocab: int = 50280,
-                 max_nodes: int = 64, act: torch.dtype = torch.bfloat16, seed: int = 0, device="cuda"):
+                 max_nodes: int = 64, act: torch.dtype = torch.bfloat16, seed: int = 0, device="cuda", fused: bool = False):
         g = torch.Generator(device=device).manual_seed(seed)
         self.n_layers, self.d_model, self.d_inner, self.dt_rank, self.vocab, self.act, self.dev = n_layers, d_model, d_inner, dt_rank, vocab, act, device
         N = 16
@@ -38,6 +40,10 @@ class ToyDrafter:
         self.W_dt = [rnd(dt_rank, d_inner, scale=dt_rank ** -0.5) for _ in range(n_layers)]
         self.W_out = [rnd(d_inner, d_model, scale=d_inner ** -0.5 / (2 * n_layers) ** 0.5) for _ in range(n_layers)]
         self.W_lm = rnd(d_model, vocab, scale=d_model ** -0.5)
+        self.fused = fused
+        if fused:   # the library takes both matrices as (out features, in features), rows contiguous
+            self.W_x_rows = [w.T.contiguous() for w in self.W_x]
+            self.W_dt_rows = [w.T.contiguous() for w in self.W_dt]
         A = -torch.arange(1, N + 1, dtype=torch.float32, device=device).repeat(d_inner, 1).contiguous()
         self.layers: List[mb.Layer] = []
         for _ in range(n_layers):
@@ -58,8 +64,7 @@ class ToyDrafter:
 
     @staticmethod
     def _norm(h: torch.Tensor) -> torch.Tensor:
-        hf = h.float()
-        return (hf * torch.rsqrt(hf.pow(2).mean(-1, keepdim=True) + 1e-5)).to(h.dtype)
+        return torch.nn.functional.rms_norm(h, (h.shape[-1],), eps=1e-5)
 
     def _generation(self, lo: int, hi: int) -> None:
         """One batch-generation step for nodes [lo, hi): tokens / parent_slot / node_slot rows lo..hi-1 are read,
@@ -71,6 +76,11 @@ class ToyDrafter:
         for l in range(self.n_layers):
             xz = self._norm(h) @ self.W_in[l]
             x, z = xz[:, :self.d_inner], xz[:, self.d_inner:]
+            if self.fused:
+                mb.mdraft_tree_step_proj(self.layers[l], self.cache, l, self.W_x_rows[l], self.W_dt_rows[l], x, z, y, ps, ns, self.status,
+                                         flags=mb.MDRAFT_DT_SOFTPLUS | mb.MDRAFT_A_POWERS)
+                h = h + y @ self.W_out[l]
+                continue
             mb.mdraft_tree_step(self.layers[l], self.cache, l, x, None, None, None, None, u, ps, ns, None, self.status,
                                 flags=mb.MDRAFT_CONV_ONLY)
             dbc = u @ self.W_x[l]

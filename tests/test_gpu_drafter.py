@@ -1,4 +1,5 @@
-"""The split mode inside a real block stack (conv step -> projections -> S6 step, states forked by slot) against an
+"""The split mode and the one-launch projection step inside a real block stack (conv step -> projections -> S6 step,
+states forked by slot) against an
 fp64 replica assembled from the oracle: every node's logits must equal those of its root-to-node token path pushed
 through the same weights layer by layer."""
 
@@ -38,8 +39,10 @@ def _replica_logits(d: ToyDrafter, path_tokens, conv0, h0):
     return (norm(h) @ f(d.W_lm))[-1]
 
 
-def test_toy_drafter_tree_matches_path_replica():
-    d = ToyDrafter(n_layers=2, d_model=32, d_inner=64, dt_rank=4, vocab=97, max_nodes=32, act=torch.float32, seed=1)
+@pytest.mark.parametrize("fused", [False, True])
+def test_toy_drafter_tree_matches_path_replica(fused):
+    d = ToyDrafter(n_layers=2, d_model=32, d_inner=64, dt_rank=8 if fused else 4, vocab=97, max_nodes=32, act=torch.float32, seed=1,
+                   fused=fused)
     g = torch.Generator(device="cuda").manual_seed(2)
     d.cache.ssm[:, 0] = torch.randn(d.cache.ssm[:, 0].shape, generator=g, device="cuda")
     d.cache.conv[:, 0] = torch.randn(d.cache.conv[:, 0].shape, generator=g, device="cuda")
