@@ -2,9 +2,11 @@
 
     python -m paper_2506_01206_b200.profile_case prefill [tokens] [layers]
     python -m paper_2506_01206_b200.profile_case tree    [layers]
+    python -m paper_2506_01206_b200.profile_case proj    [nodes] [layers]
 
 `prefill` encodes a 130M-shaped context (default 2048 tokens x 1536 channels, bf16, 4 layers) three times;
-`tree` runs one batched-serving draft round (32 sequences x 32-node trees, default 4 layers) twice.  Both hold well
+`tree` runs one batched-serving draft round (32 sequences x 32-node trees, default 4 layers) twice; `proj` runs one
+tree level (default 18 nodes, the paper's widest, 24 layers) through the step that forms dt, B, C itself.  All hold well
 under 1 GB on the device and launch a few dozen kernels, which keeps a multi-pass profiler capture short; inputs are
 larger than L2 across the layers, so DRAM counters still mean something.
 """
@@ -73,6 +75,24 @@ def tree(n_layers: int = 4, reps: int = 2) -> None:
     print("tree: %d nodes, levels %s, %d layers x %d, status %d" % (M, np.diff(lvl).tolist(), n_layers, reps, int(status.item())))
 
 
+def proj(n_nodes: int = 18, n_layers: int = 24, reps: int = 3, dt_rank: int = 48) -> None:
+    cfg = gen.get_config(1)
+    tdt, D = torch_act(cfg.act), cfg.d_inner
+    lays = [upload_layer(gen.layer_params(cfg, l), cfg.act, FLAGS) for l in range(n_layers)]
+    Ws = [[to_device(w, tdt) for w in gen.select_proj(cfg, l, dt_rank)] for l in range(n_layers)]
+    ins = [[to_device(a, tdt) for a in gen.node_inputs(cfg, l, 0, n_nodes)[:2]] for l in range(n_layers)]
+    out = torch.empty((n_nodes, D), dtype=tdt, device="cuda")
+    cache = md.StateCache(n_layers, 1 + n_nodes, D, act=tdt)
+    cache.ssm.normal_()
+    cache.conv.normal_()
+    par, nod, status = i32([0] * n_nodes), i32(list(range(1, n_nodes + 1))), torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(reps):
+        for l in range(n_layers):
+            md.mdraft_tree_step_proj(lays[l], cache, l, Ws[l][0], Ws[l][1], ins[l][0], ins[l][1], out, par, nod, status)
+    torch.cuda.synchronize()
+    print("proj: %d nodes x %d channels, dt_rank %d, %d layers x %d, status %d" % (n_nodes, D, dt_rank, n_layers, reps, int(status.item())))
+
+
 if __name__ == "__main__":
     what = sys.argv[1] if len(sys.argv) > 1 else "prefill"
     nums = [int(v) for v in sys.argv[2:]]
@@ -80,5 +100,7 @@ if __name__ == "__main__":
         prefill(*nums)
     elif what == "tree":
         tree(*nums)
+    elif what == "proj":
+        proj(*nums)
     else:
         raise SystemExit(__doc__)
