@@ -231,6 +231,8 @@ int mdraft_tree_step(const mdraft_layer *layer, const mdraft_cache *cache, int32
  *
  *   proj->W_x, proj->W_dt : device, activation dtype of the layer, 16-byte aligned, dense (no padding)
  *   proj->dt_rank         : multiple of 8, 8..256
+ *   proj->nodes_per_cluster: tuning only (the result of a node does not depend on it, bit for bit); 0 lets the
+ *                           library choose: 1 for narrow levels, 2 or 4 for wide ones
  *   x, z, out             : device, n_nodes rows of d_inner activations (strides ldx, ldz, ldo in elements)
  *   parent_slot, node_slot: device, n_nodes int32 each; same meaning and hazards as mdraft_tree_step
  * layer->flags: MDRAFT_DT_SOFTPLUS and MDRAFT_A_POWERS are honoured; MDRAFT_PRECONV and
@@ -242,7 +244,7 @@ typedef struct mdraft_select_proj {
     const void *W_x;
     const void *W_dt;
     int32_t dt_rank;
-    int32_t reserved;   /* 0 */
+    int32_t nodes_per_cluster;   /* 0 = chosen from the level's width; 1, 2 or 4 = that many nodes share one set of weight loads */
 } mdraft_select_proj;
 
 int mdraft_tree_step_proj(const mdraft_layer *layer, const mdraft_cache *cache, int32_t layer_index,

@@ -55,7 +55,7 @@ class _PrefillOpts(C.Structure):
 
 
 class _SelectProj(C.Structure):
-    _fields_ = [("W_x", C.c_void_p), ("W_dt", C.c_void_p), ("dt_rank", C.c_int32), ("reserved", C.c_int32)]
+    _fields_ = [("W_x", C.c_void_p), ("W_dt", C.c_void_p), ("dt_rank", C.c_int32), ("nodes_per_cluster", C.c_int32)]
 
 
 class _Ucb(C.Structure):
@@ -310,7 +310,8 @@ def mdraft_tree_step(layer: Layer, cache: StateCache, layer_index: int, x, z, dt
 
 def mdraft_tree_step_proj(layer: Layer, cache: StateCache, layer_index: int, W_x: torch.Tensor, W_dt: torch.Tensor,
                           x, z, out, parent_slot: torch.Tensor, node_slot: torch.Tensor,
-                          dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None) -> None:
+                          dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None,
+                          nodes_per_cluster: int = 0) -> None:
     """One tree level where dt, B and C come from the block's projections of the conv output.
     W_x: (dt_rank + 2 N, D) and W_dt: (D, dt_rank), contiguous, in the layer's activation dtype."""
     lib = load_library()
@@ -327,7 +328,7 @@ def mdraft_tree_step_proj(layer: Layer, cache: StateCache, layer_index: int, W_x
     R = int(W_dt.shape[1])
     if tuple(W_dt.shape) != (layer.d_inner, R) or tuple(W_x.shape) != (R + 2 * layer.d_state, layer.d_inner):
         raise ValueError("W_x must be (dt_rank + 2 d_state, d_inner) and W_dt (d_inner, dt_rank)")
-    pr = _SelectProj(W_x.data_ptr(), W_dt.data_ptr(), R, 0)
+    pr = _SelectProj(W_x.data_ptr(), W_dt.data_ptr(), R, int(nodes_per_cluster))
     rc = lib.mdraft_tree_step_proj(C.byref(cl), C.byref(cc), int(layer_index), C.byref(pr), px, ldx, pz, ldz, po, ldo,
                                    M, _ptr(parent_slot), _ptr(node_slot), _ptr(dev_status), _stream_ptr(stream))
     if rc != 0:

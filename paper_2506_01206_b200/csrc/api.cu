@@ -310,6 +310,8 @@ int mdraft_tree_step_proj(const mdraft_layer* layer, const mdraft_cache* cache, 
     if (!aligned16(proj->W_x) || !aligned16(proj->W_dt)) return MDRAFT_ERR_MISALIGNED;
     if (proj->dt_rank < 8 || proj->dt_rank > kProjMaxRank || (proj->dt_rank % 8) != 0) return MDRAFT_ERR_UNSUPPORTED;
     if (tree_proj_block_channels(layer->d_inner) == 0) return MDRAFT_ERR_UNSUPPORTED;
+    if (proj->nodes_per_cluster != 0 && proj->nodes_per_cluster != 1 && proj->nodes_per_cluster != 2 && proj->nodes_per_cluster != 4)
+        return MDRAFT_ERR_INVALID_ARG;
     if (n_nodes == 0) return MDRAFT_OK;
     if (!parent_slot || !node_slot) return MDRAFT_ERR_INVALID_ARG;
     const int D = layer->d_inner, act = layer->act;
@@ -322,7 +324,7 @@ int mdraft_tree_step_proj(const mdraft_layer* layer, const mdraft_cache* cache, 
     a.pool = pool_dev(cache, act, layer_index);
     a.x = x; a.z = z; a.out = out;
     a.ldx = ldx; a.ldz = ldz; a.ldo = ldo;
-    a.W_x = proj->W_x; a.W_dt = proj->W_dt; a.dt_rank = proj->dt_rank;
+    a.W_x = proj->W_x; a.W_dt = proj->W_dt; a.dt_rank = proj->dt_rank; a.nodes_per_cluster = proj->nodes_per_cluster;
     a.parent_slot = parent_slot; a.node_slot = node_slot; a.n_nodes = n_nodes; a.dev_status = dev_status;
     if (launch_tree_proj(a, act, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MDRAFT_ERR_CUDA;
     return MDRAFT_OK;

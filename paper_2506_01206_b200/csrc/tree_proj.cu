@@ -120,52 +120,86 @@ __device__ __forceinline__ float dot4(const float4& a, const float4& b, float ac
     return acc;
 }
 
-template <typename AT, int CB, bool kPow>
+// Shared-memory layout of a block: NT nodes x CB channels.  Byte offsets into the dynamic array; all multiples of 16.
+template <typename AT, int CB, int NT>
+struct ProjSmem {
+    static constexpr int kH = 0;                                           // [NT][CB][16] fp32 state slices
+    static constexpr int kConv = kH + NT * CB * kN * 4;                    // [NT][W-1][CB] window rows
+    static constexpr int kX = kConv + NT * (kW - 1) * CB * (int)sizeof(AT);  // [NT][CB] x rows; receive the out rows
+    static constexpr int kZ = kX + NT * CB * (int)sizeof(AT);              // [NT][CB] z rows
+    static constexpr int kU = kZ + NT * CB * (int)sizeof(AT);              // [NT][CB] fp32 conv outputs
+    static constexpr int kPart = kU + NT * CB * 4;                         // [NT][kMaxRows] this block's share of s
+    static constexpr int kS = kPart + NT * kMaxRows * 4;                   // [NT][kMaxRows] s, summed over the cluster
+    static constexpr int kBars = kS + NT * kMaxRows * 4;                   // [NT][2] mbarriers
+    static constexpr int kTotal = kBars + NT * 2 * 8;
+};
+
+// A block is CB channels of NT consecutive nodes of the level; the blocks that cover one such group of nodes form
+// the cluster.  With NT > 1 the rows of W_x and W_dt a thread holds serve NT nodes, which is what wide levels need
+// (every node otherwise re-reads both matrices out of L2).
+template <typename AT, int CB, int NT, bool kPow>
 __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
     constexpr int NW = CB / 32;    // warps
     constexpr int NP = CB / 128;   // a lane owns 4 consecutive channels in each of NP 128-channel spans
-    __shared__ __align__(128) float4 s_h[CB * (kN / 4)];  // state slice [channel][quad]
-    __shared__ __align__(16) AT s_conv[kW - 1][CB];
-    __shared__ __align__(16) AT s_x[CB];                  // the node's x row; receives the out row afterwards
-    __shared__ __align__(16) AT s_z[CB];
-    __shared__ __align__(16) float s_u[CB];               // conv outputs of this block's channels
-    __shared__ __align__(16) float s_part[kMaxRows];      // this block's share of s = W_x u
-    __shared__ __align__(16) float s_s[kMaxRows];         // s, summed over the cluster
-    __shared__ __align__(8) uint64_t bar_a, bar_b;
+    using S = ProjSmem<AT, CB, NT>;
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    float4* const s_h = reinterpret_cast<float4*>(s_dyn + S::kH);
+    AT* const s_conv = reinterpret_cast<AT*>(s_dyn + S::kConv);
+    AT* const s_x = reinterpret_cast<AT*>(s_dyn + S::kX);
+    AT* const s_z = reinterpret_cast<AT*>(s_dyn + S::kZ);
+    float* const s_u = reinterpret_cast<float*>(s_dyn + S::kU);
+    float* const s_part = reinterpret_cast<float*>(s_dyn + S::kPart);
+    float* const s_s = reinterpret_cast<float*>(s_dyn + S::kS);
+    uint64_t* const bars = reinterpret_cast<uint64_t*>(s_dyn + S::kBars);  // [i][0]: x + window, [i][1]: z + state
 
     const int D = p.L.d_inner, R = p.dt_rank, rows = R + 2 * kN;
-    const int node = blockIdx.x;
+    const int node0 = blockIdx.x * NT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int d0 = blockIdx.y * CB;
     const int cols = min(CB, D - d0);
     const int d = d0 + tid;
     const bool live = tid < cols;
-    const int pslot = __ldg(p.parent_slot + node);
-    const int nslot = __ldg(p.node_slot + node);
-    // The slots are the node's, so every block of the cluster takes the same way out here, before any barrier.
-    if (pslot < -1 || pslot >= p.pool.n_slots || nslot < 0 || nslot >= p.pool.n_slots) {
-        if (tid == 0 && blockIdx.y == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
-        return;
-    }
     const uint32_t flags = p.L.flags;
-    const bool have_parent = pslot >= 0;
     const uint32_t row_bytes = (uint32_t)cols * sizeof(AT), h_bytes = (uint32_t)cols * kN * 4u;
-    float* h_parent = p.pool.ssm + (size_t)pslot * p.pool.ssm_slot_stride + (size_t)d0 * kN;
-    float* h_child = p.pool.ssm + (size_t)nslot * p.pool.ssm_slot_stride + (size_t)d0 * kN;
-    AT* conv_parent = static_cast<AT*>(p.pool.conv) + (size_t)pslot * p.pool.conv_slot_stride + d0;
-    AT* conv_child = static_cast<AT*>(p.pool.conv) + (size_t)nslot * p.pool.conv_slot_stride + d0;
+
+    // Slots of this block's nodes.  They are the nodes', not the block's, so every block of the cluster decides
+    // alike; a node with a slot out of range is skipped (nothing loaded, nothing stored) but nobody leaves early.
+    int pslot[NT], nslot[NT];
+    bool valid[NT];
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+        valid[i] = node0 + i < p.n_nodes;
+        pslot[i] = valid[i] ? __ldg(p.parent_slot + node0 + i) : -1;
+        nslot[i] = valid[i] ? __ldg(p.node_slot + node0 + i) : 0;
+        if (valid[i] && (pslot[i] < -1 || pslot[i] >= p.pool.n_slots || nslot[i] < 0 || nslot[i] >= p.pool.n_slots)) {
+            valid[i] = false;
+            if (tid == 0 && blockIdx.y == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+        }
+    }
 
     if (tid == 0) {
-        mbar_init(&bar_a, 1);
-        mbar_init(&bar_b, 1);
+#pragma unroll
+        for (int i = 0; i < 2 * NT; ++i) mbar_init(&bars[i], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        mbar_expect_tx(&bar_a, row_bytes + (have_parent ? (kW - 1) * row_bytes : 0u));
-        bulk_load(s_x, static_cast<const AT*>(p.x) + (size_t)node * p.ldx + d0, row_bytes, &bar_a);
-        if (have_parent)
-            for (int j = 0; j < kW - 1; ++j) bulk_load(s_conv[j], conv_parent + (size_t)j * D, row_bytes, &bar_a);
-        mbar_expect_tx(&bar_b, row_bytes + (have_parent ? h_bytes : 0u));
-        if (have_parent) bulk_load(s_h, h_parent, h_bytes, &bar_b);
-        bulk_load(s_z, static_cast<const AT*>(p.z) + (size_t)node * p.ldz + d0, row_bytes, &bar_b);
+#pragma unroll
+        for (int i = 0; i < NT; ++i) {
+            if (!valid[i]) continue;
+            const bool have_parent = pslot[i] >= 0;
+            const AT* conv_parent = static_cast<const AT*>(p.pool.conv) + (size_t)pslot[i] * p.pool.conv_slot_stride + d0;
+            mbar_expect_tx(&bars[2 * i], row_bytes + (have_parent ? (kW - 1) * row_bytes : 0u));
+            bulk_load(s_x + i * CB, static_cast<const AT*>(p.x) + (size_t)(node0 + i) * p.ldx + d0, row_bytes, &bars[2 * i]);
+            if (have_parent)
+                for (int j = 0; j < kW - 1; ++j) bulk_load(s_conv + (i * (kW - 1) + j) * CB, conv_parent + (size_t)j * D, row_bytes, &bars[2 * i]);
+        }
+#pragma unroll
+        for (int i = 0; i < NT; ++i) {
+            if (!valid[i]) continue;
+            const bool have_parent = pslot[i] >= 0;
+            mbar_expect_tx(&bars[2 * i + 1], row_bytes + (have_parent ? h_bytes : 0u));
+            if (have_parent)
+                bulk_load(s_h + i * CB * (kN / 4), p.pool.ssm + (size_t)pslot[i] * p.pool.ssm_slot_stride + (size_t)d0 * kN, h_bytes, &bars[2 * i + 1]);
+            bulk_load(s_z + i * CB, static_cast<const AT*>(p.z) + (size_t)(node0 + i) * p.ldz + d0, row_bytes, &bars[2 * i + 1]);
+        }
     }
 
     // Layer constants travel by ordinary loads while the copies are in flight.
@@ -189,6 +223,7 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
     }
     // The weights depend on nothing that is still in flight: the first rows of this warp's share of W_x and the
     // head of this channel's row of W_dt are requested now, ahead of the waits they would otherwise queue behind.
+    // (Giving the registers up for more resident blocks on wide levels was measured: it is slower at every width.)
     constexpr int kPreRows = NP == 4 ? (sizeof(AT) == 4 ? 3 : 5) : 10;  // rows of W_x held in registers per warp
     constexpr int kPreDt = sizeof(AT) == 4 ? 3 : 6;  // groups of eight weights of W_dt held in registers per thread
     const AT* wx = static_cast<const AT*>(p.W_x) + d0 + 4 * lane;
@@ -212,75 +247,101 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
         dpre[j].load(wr + (8 * j < R ? 8 * j : 0));
 
     __syncthreads();  // the mbarriers are initialised for everyone
-    bool bad = __syncthreads_or(!mbar_wait_bounded(&bar_a, 0u));
-
-    // ---- conv window: (w0, w1, w2, x) -> (w1, w2, x)
-    float u = 0.f;
-    if (live && !bad) {
-        const float xv = Act<AT>::to_f32(s_x[tid]);
-        float win[kW - 1] = {0.f, 0.f, 0.f};
-        if (have_parent) {
+    bool waited = true;
 #pragma unroll
-            for (int j = 0; j < kW - 1; ++j) win[j] = Act<AT>::to_f32(s_conv[j][tid]);
+    for (int i = 0; i < NT; ++i)
+        if (valid[i]) waited = mbar_wait_bounded(&bars[2 * i], 0u) && waited;
+    bool bad = __syncthreads_or(!waited);
+
+    // ---- conv window of every node: (w0, w1, w2, x) -> (w1, w2, x)
+    float u[NT];
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+        u[i] = 0.f;
+        if (live && !bad && valid[i]) {
+            AT* cw = s_conv + i * (kW - 1) * CB + tid;
+            const float xv = Act<AT>::to_f32(s_x[i * CB + tid]);
+            float win[kW - 1] = {0.f, 0.f, 0.f};
+            if (pslot[i] >= 0) {
+#pragma unroll
+                for (int j = 0; j < kW - 1; ++j) win[j] = Act<AT>::to_f32(cw[j * CB]);
+            }
+            float acc = fmaf(wv.x, win[0], cb);
+            acc = fmaf(wv.y, win[1], acc);
+            acc = fmaf(wv.z, win[2], acc);
+            acc = fmaf(wv.w, xv, acc);
+            u[i] = silu(acc);
+            cw[0] = Act<AT>::from_f32(win[1]);
+            cw[CB] = Act<AT>::from_f32(win[2]);
+            cw[2 * CB] = Act<AT>::from_f32(xv);
         }
-        float acc = fmaf(wv.x, win[0], cb);
-        acc = fmaf(wv.y, win[1], acc);
-        acc = fmaf(wv.z, win[2], acc);
-        acc = fmaf(wv.w, xv, acc);
-        u = silu(acc);
-        s_conv[0][tid] = Act<AT>::from_f32(win[1]);
-        s_conv[1][tid] = Act<AT>::from_f32(win[2]);
-        s_conv[2][tid] = Act<AT>::from_f32(xv);
+        s_u[i * CB + tid] = u[i];
     }
-    s_u[tid] = u;
     __syncthreads();
 
-    // ---- this block's share of s = W_x u: a warp takes every NW-th row, a lane 4 NP channels of it.
+    // ---- this block's share of s = W_x u per node: a warp takes every NW-th row, a lane 4 NP channels of it.
     {
-        float4 uu[NP];
+        float4 uu[NT][NP];
 #pragma unroll
-        for (int q = 0; q < NP; ++q) uu[q] = *reinterpret_cast<const float4*>(&s_u[q * 128 + 4 * lane]);
-        float acc[kPreRows];
+        for (int i = 0; i < NT; ++i)
+#pragma unroll
+            for (int q = 0; q < NP; ++q) uu[i][q] = *reinterpret_cast<const float4*>(&s_u[i * CB + q * 128 + 4 * lane]);
+        float acc[NT][kPreRows];
 #pragma unroll
         for (int j = 0; j < kPreRows; ++j) {
-            acc[j] = 0.f;
+            float4 wq[NP];
 #pragma unroll
-            for (int q = 0; q < NP; ++q)
-                if (in[q]) acc[j] = dot4(wpre[j][q].get(), uu[q], acc[j]);
+            for (int q = 0; q < NP; ++q) wq[q] = wpre[j][q].get();
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                acc[i][j] = 0.f;
+#pragma unroll
+                for (int q = 0; q < NP; ++q)
+                    if (in[q]) acc[i][j] = dot4(wq[q], uu[i][q], acc[i][j]);
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-            for (int j = 0; j < kPreRows; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+            for (int i = 0; i < NT; ++i)
+#pragma unroll
+                for (int j = 0; j < kPreRows; ++j) acc[i][j] += __shfl_xor_sync(0xffffffffu, acc[i][j], o);
         }
         if (lane == 0) {
 #pragma unroll
-            for (int j = 0; j < kPreRows; ++j)
-                if (warp + j * NW < rows) s_part[warp + j * NW] = acc[j];
+            for (int i = 0; i < NT; ++i)
+#pragma unroll
+                for (int j = 0; j < kPreRows; ++j)
+                    if (warp + j * NW < rows) s_part[i * kMaxRows + warp + j * NW] = acc[i][j];
         }
-        // Rows beyond the prefetched ones (large dt_rank), four in flight per warp.
+        // Rows beyond the prefetched ones (large dt_rank), four rows of W_x in flight per warp.
         constexpr int kBatch = 4;
         for (int r0 = warp + kPreRows * NW; r0 < rows; r0 += kBatch * NW) {
-            float a4[kBatch];
+            float4 wq[kBatch][NP];
 #pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                const int r = r0 + j * NW;
-                a4[j] = 0.f;
-                if (r < rows) {
+            for (int j = 0; j < kBatch; ++j)
 #pragma unroll
-                    for (int q = 0; q < NP; ++q)
-                        if (in[q]) a4[j] = dot4(load_w4(wx + (size_t)r * D + q * 128), uu[q], a4[j]);
+                for (int q = 0; q < NP; ++q)
+                    wq[j][q] = (r0 + j * NW < rows && in[q]) ? load_w4(wx + (size_t)(r0 + j * NW) * D + q * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                float a4[kBatch];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    a4[j] = 0.f;
+#pragma unroll
+                    for (int q = 0; q < NP; ++q) a4[j] = dot4(wq[j][q], uu[i][q], a4[j]);
                 }
-            }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
+                for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-                for (int j = 0; j < kBatch; ++j) a4[j] += __shfl_xor_sync(0xffffffffu, a4[j], o);
-            }
-            if (lane == 0) {
+                    for (int j = 0; j < kBatch; ++j) a4[j] += __shfl_xor_sync(0xffffffffu, a4[j], o);
+                }
+                if (lane == 0) {
 #pragma unroll
-                for (int j = 0; j < kBatch; ++j)
-                    if (r0 + j * NW < rows) s_part[r0 + j * NW] = a4[j];
+                    for (int j = 0; j < kBatch; ++j)
+                        if (r0 + j * NW < rows) s_part[i * kMaxRows + r0 + j * NW] = a4[j];
+                }
             }
         }
     }
@@ -289,49 +350,70 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
     cluster_wait();
     {
         const uint32_t nblk = cluster_size();
-        for (int r = tid; r < rows; r += CB) {
+        for (int idx = tid; idx < NT * rows; idx += CB) {
+            const int i = idx / rows, r = idx - i * rows;
             float sum = 0.f;
-            for (uint32_t c = 0; c < nblk; ++c) sum += peer_block_float(&s_part[r], c);
-            s_s[r] = sum;
+            for (uint32_t c = 0; c < nblk; ++c) sum += peer_block_float(&s_part[i * kMaxRows + r], c);
+            s_s[i * kMaxRows + r] = sum;
         }
     }
     cluster_arrive();  // this block no longer reads its neighbours; the matching wait is the last thing it does
     __syncthreads();
 
-    // ---- step size of this thread's channel: dt = W_dt[d][:] . s[0:R]  (R is a multiple of 8)
-    float dtv = 0.f;
+    // ---- step size of this thread's channel in every node: dt = W_dt[d][:] . s[0:R]  (R is a multiple of 8)
+    float dtv[NT];
+#pragma unroll
+    for (int i = 0; i < NT; ++i) dtv[i] = 0.f;
     if (live) {
-        float acc0 = 0.f, acc1 = 0.f;
+        float acc0[NT], acc1[NT];
+#pragma unroll
+        for (int i = 0; i < NT; ++i) { acc0[i] = 0.f; acc1[i] = 0.f; }
 #pragma unroll
         for (int j = 0; j < kPreDt; ++j) {
             if (8 * j < R) {
-                acc0 = dot4(dpre[j].lo(), *reinterpret_cast<const float4*>(&s_s[8 * j]), acc0);
-                acc1 = dot4(dpre[j].hi(), *reinterpret_cast<const float4*>(&s_s[8 * j + 4]), acc1);
+                const float4 w0 = dpre[j].lo(), w1 = dpre[j].hi();
+#pragma unroll
+                for (int i = 0; i < NT; ++i) {
+                    acc0[i] = dot4(w0, *reinterpret_cast<const float4*>(&s_s[i * kMaxRows + 8 * j]), acc0[i]);
+                    acc1[i] = dot4(w1, *reinterpret_cast<const float4*>(&s_s[i * kMaxRows + 8 * j + 4]), acc1[i]);
+                }
             }
         }
 #pragma unroll 2
         for (int r = 8 * kPreDt; r < R; r += 8) {
             const float4 w0 = load_w4(wr + r), w1 = load_w4(wr + r + 4);
-            acc0 = dot4(w0, *reinterpret_cast<const float4*>(&s_s[r]), acc0);
-            acc1 = dot4(w1, *reinterpret_cast<const float4*>(&s_s[r + 4]), acc1);
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                acc0[i] = dot4(w0, *reinterpret_cast<const float4*>(&s_s[i * kMaxRows + r]), acc0[i]);
+                acc1[i] = dot4(w1, *reinterpret_cast<const float4*>(&s_s[i * kMaxRows + r + 4]), acc1[i]);
+            }
         }
-        dtv = acc0 + acc1;
+#pragma unroll
+        for (int i = 0; i < NT; ++i) dtv[i] = acc0[i] + acc1[i];
     }
 
-    bad = __syncthreads_or(bad || !mbar_wait_bounded(&bar_b, 0u));
+    waited = true;
+#pragma unroll
+    for (int i = 0; i < NT; ++i)
+        if (valid[i]) waited = mbar_wait_bounded(&bars[2 * i + 1], 0u) && waited;
+    bad = __syncthreads_or(bad || !waited);
 
-    if (live && !bad) {
+#pragma unroll
+    for (int i = 0; i < NT; ++i) {
+        if (!(live && !bad && valid[i])) continue;
         // ---- one step of the recurrence.  The quads of a channel are visited in an order that differs between
         // neighbouring threads, which keeps the 128-bit shared-memory accesses free of bank conflicts.
+        float4* hs = s_h + (i * CB + tid) * (kN / 4);
+        const float* ss = s_s + i * kMaxRows;
         const int sw = (tid >> 1) & 3;
         float4 hq[kN / 4];
 #pragma unroll
-        for (int i = 0; i < kN / 4; ++i) hq[i] = have_parent ? s_h[tid * (kN / 4) + (i ^ sw)] : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k = 0; k < kN / 4; ++k) hq[k] = pslot[i] >= 0 ? hs[k ^ sw] : make_float4(0.f, 0.f, 0.f, 0.f);
         xor_permute(hq, sw);
-        const float zv = Act<AT>::to_f32(s_z[tid]);
-        const float v = dtv + dtb;
+        const float zv = Act<AT>::to_f32(s_z[i * CB + tid]);
+        const float v = dtv[i] + dtb;
         const float delta = (flags & MDRAFT_DT_SOFTPLUS) ? softplus(v) : v;
-        const float du = delta * u;
+        const float du = delta * u[i];
         float P[kN];
         if constexpr (kPow) {
             const float r1 = ex2(delta * a2[0]);
@@ -348,8 +430,8 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
 #pragma unroll
         for (int q = 0; q < kN / 4; ++q) {
             h[4 * q] = hq[q].x; h[4 * q + 1] = hq[q].y; h[4 * q + 2] = hq[q].z; h[4 * q + 3] = hq[q].w;
-            const float4 b = *reinterpret_cast<const float4*>(&s_s[R + 4 * q]);
-            const float4 c = *reinterpret_cast<const float4*>(&s_s[R + kN + 4 * q]);
+            const float4 b = *reinterpret_cast<const float4*>(&ss[R + 4 * q]);
+            const float4 c = *reinterpret_cast<const float4*>(&ss[R + kN + 4 * q]);
             Bv[4 * q] = b.x; Bv[4 * q + 1] = b.y; Bv[4 * q + 2] = b.z; Bv[4 * q + 3] = b.w;
             Cv[4 * q] = c.x; Cv[4 * q + 1] = c.y; Cv[4 * q + 2] = c.z; Cv[4 * q + 3] = c.w;
         }
@@ -363,23 +445,29 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
         for (int q = 0; q < kN / 4; ++q) hq[q] = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
         xor_permute(hq, sw);
 #pragma unroll
-        for (int i = 0; i < kN / 4; ++i) s_h[tid * (kN / 4) + (i ^ sw)] = hq[i];
-        s_x[tid] = Act<AT>::from_f32(fmaf(dsk, u, y0 + y1) * silu(zv));
+        for (int k = 0; k < kN / 4; ++k) hs[k ^ sw] = hq[k];
+        s_x[i * CB + tid] = Act<AT>::from_f32(fmaf(dsk, u[i], y0 + y1) * silu(zv));
     }
     // Shared-memory writes above must be visible to the copy engine before it reads them.
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
     if (tid == 0) {
         if (bad) {
-            // Nothing of this node is stored.  The copies target this block's shared memory: give them one more
+            // Nothing of these nodes is stored.  The copies target this block's shared memory: give them one more
             // bounded chance to land before the block ends.
             flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
-            mbar_wait_bounded(&bar_a, 0u);
-            mbar_wait_bounded(&bar_b, 0u);
+#pragma unroll
+            for (int i = 0; i < NT; ++i)
+                if (valid[i]) { mbar_wait_bounded(&bars[2 * i], 0u); mbar_wait_bounded(&bars[2 * i + 1], 0u); }
         } else {
-            bulk_store(h_child, s_h, h_bytes);
-            for (int j = 0; j < kW - 1; ++j) bulk_store(conv_child + (size_t)j * D, s_conv[j], row_bytes);
-            bulk_store(static_cast<AT*>(p.out) + (size_t)node * p.ldo + d0, s_x, row_bytes);
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                if (!valid[i]) continue;
+                bulk_store(p.pool.ssm + (size_t)nslot[i] * p.pool.ssm_slot_stride + (size_t)d0 * kN, s_h + i * CB * (kN / 4), h_bytes);
+                AT* conv_child = static_cast<AT*>(p.pool.conv) + (size_t)nslot[i] * p.pool.conv_slot_stride + d0;
+                for (int j = 0; j < kW - 1; ++j) bulk_store(conv_child + (size_t)j * D, s_conv + (i * (kW - 1) + j) * CB, row_bytes);
+                bulk_store(static_cast<AT*>(p.out) + (size_t)(node0 + i) * p.ldo + d0, s_x + i * CB, row_bytes);
+            }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory stays valid until it has been read
         }
@@ -388,32 +476,43 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
     cluster_wait();  // no block of the cluster leaves while a neighbour may still read its share of s
 }
 
-template <typename AT, int CB>
-cudaError_t launch_cb(const TreeProjArgs& p, int n_blocks, cudaStream_t st) {
+template <typename AT, int CB, int NT>
+cudaError_t launch_nt(const TreeProjArgs& p, int n_blocks, cudaStream_t st) {
+    constexpr int kSmem = ProjSmem<AT, CB, NT>::kTotal;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)p.n_nodes, (unsigned)n_blocks, 1);
+    cfg.gridDim = dim3((unsigned)((p.n_nodes + NT - 1) / NT), (unsigned)n_blocks, 1);
     cfg.blockDim = dim3(CB, 1, 1);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = kSmem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 1;
-    at[0].val.clusterDim.y = (unsigned)n_blocks;  // the blocks of one node
+    at[0].val.clusterDim.y = (unsigned)n_blocks;  // the blocks of one group of nodes
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    if (p.L.flags & MDRAFT_A_POWERS) return cudaLaunchKernelEx(&cfg, tree_proj_kernel<AT, CB, true>, p);
-    return cudaLaunchKernelEx(&cfg, tree_proj_kernel<AT, CB, false>, p);
+    const bool pow = p.L.flags & MDRAFT_A_POWERS;
+    auto kernel = pow ? tree_proj_kernel<AT, CB, NT, true> : tree_proj_kernel<AT, CB, NT, false>;
+    if (kSmem > 48 * 1024) {  // a property of the loaded function, not an allocation
+        const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
 template <typename AT>
 cudaError_t launch_act(const TreeProjArgs& p, cudaStream_t st) {
     const int cb = tree_proj_block_channels(p.L.d_inner);
     const int n_blocks = (p.L.d_inner + cb - 1) / cb;
+    // Nodes per cluster: one while the level is narrow (latency is what counts and every node gets its own SMs);
+    // two or four once the level is wide enough that re-reading the two matrices per node is what costs.
+    int nt = p.nodes_per_cluster;
+    if (nt <= 0) nt = p.n_nodes * n_blocks <= 2 * 148 ? 1 : (p.n_nodes * n_blocks <= 4 * 148 ? 2 : 4);
+    if (cb == 512) nt = 1;  // the widest block has no registers to spare for a second node
     switch (cb) {
-        case 128: return launch_cb<AT, 128>(p, n_blocks, st);
-        case 256: return launch_cb<AT, 256>(p, n_blocks, st);
-        case 512: return launch_cb<AT, 512>(p, n_blocks, st);
+        case 128: return nt == 1 ? launch_nt<AT, 128, 1>(p, n_blocks, st) : nt == 2 ? launch_nt<AT, 128, 2>(p, n_blocks, st) : launch_nt<AT, 128, 4>(p, n_blocks, st);
+        case 256: return nt == 1 ? launch_nt<AT, 256, 1>(p, n_blocks, st) : nt == 2 ? launch_nt<AT, 256, 2>(p, n_blocks, st) : launch_nt<AT, 256, 4>(p, n_blocks, st);
+        case 512: return launch_nt<AT, 512, 1>(p, n_blocks, st);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -17,6 +17,7 @@ struct TreeProjArgs {
     const void* W_x;   // (dt_rank + 2 N, D) row-major
     const void* W_dt;  // (D, dt_rank) row-major
     int dt_rank;
+    int nodes_per_cluster;  // 0: chosen from the level's width; else 1, 2 or 4
     const int32_t *parent_slot, *node_slot;
     int n_nodes;
     int32_t* dev_status;

@@ -19,8 +19,8 @@ from paper_2506_01206_b200.device_inputs import i32, to_device, torch_act, uploa
 class ProjRig:
     """One layer, one sequence: committed state in slot 0, node i in slot 1+i."""
 
-    def __init__(self, cfg, tree, dt_rank, conv_bias=True, general_A=True, flags=md.MDRAFT_DT_SOFTPLUS, seed_state=5):
-        self.cfg, self.tree, self.flags = cfg, tree, flags
+    def __init__(self, cfg, tree, dt_rank, conv_bias=True, general_A=True, flags=md.MDRAFT_DT_SOFTPLUS, seed_state=5, nodes_per_cluster=0):
+        self.cfg, self.tree, self.flags, self.nodes_per_cluster = cfg, tree, flags, nodes_per_cluster
         self.tdt = torch_act(cfg.act)
         self.params = gen.layer_params(cfg, 0, conv_bias=conv_bias, general_A=general_A)
         self.lay = upload_layer(self.params, cfg.act, flags)
@@ -48,7 +48,8 @@ class ProjRig:
         t = torch.from_numpy(np.asarray(idx)).cuda()
         out = torch.full((len(idx), self.cfg.d_inner), float("nan"), dtype=self.tdt, device="cuda")
         md.mdraft_tree_step_proj(self.lay, self.cache, 0, self.dW_x, self.dW_dt, self.dx[t].contiguous(), self.dz[t].contiguous(),
-                                 out, i32(self.parent_slot[idx]), i32(self.node_slot[idx]), self.status)
+                                 out, i32(self.parent_slot[idx]), i32(self.node_slot[idx]), self.status,
+                                 nodes_per_cluster=self.nodes_per_cluster)
         torch.cuda.synchronize()
         return out
 
@@ -109,6 +110,38 @@ def test_structured_A_fast_path_and_plain_step_size(act):
         assert_close(rig.states()[0], o_h, TOL_STATE, f"node SSM states (flags {flags})")
 
 
+@pytest.mark.parametrize("act,Dn,R", [("bf16", 1536, 48), ("f32", 200, 16), ("bf16", 1024, 96), ("f32", 2048, 64)])
+def test_nodes_per_cluster_changes_no_bit_and_matches_oracle(act, Dn, R):
+    """Levels of 1, 3, 9, 18 nodes (ragged against groups of 2 and 4) with 1, 2 and 4 nodes per cluster."""
+    cfg = parity.small_config(Dn, act)
+    tree = gen.paper_tree((3, 3, 2))
+    ref = None
+    for npc in (1, 2, 4):
+        rig = ProjRig(cfg, tree, R, nodes_per_cluster=npc)
+        out = rig.run_levels()
+        assert int(rig.status.item()) == 0
+        h, conv = rig.states()
+        if ref is None:
+            ref = (out, h, conv)
+            o_out, o_conv, o_h, _, _, _ = rig.oracle()
+            assert_close(out.float().cpu().numpy(), o_out, TOL[act], "node outputs")
+            assert_close(h, o_h, TOL_STATE, "node SSM states")
+        else:
+            assert torch.equal(out, ref[0]) and np.array_equal(h, ref[1]) and np.array_equal(conv, ref[2]), f"{npc} nodes per cluster"
+
+
+def test_wide_level_takes_the_grouped_path_by_itself():
+    """300 children of the committed state: the library's own choice groups nodes; every node still equals the oracle's."""
+    cfg = parity.small_config(1536, "bf16")
+    tree = gen.full_tree([300])
+    rig = ProjRig(cfg, tree, 48, general_A=False, flags=md.MDRAFT_DT_SOFTPLUS | md.MDRAFT_A_POWERS)
+    out = rig.run_levels()
+    assert int(rig.status.item()) == 0
+    o_out, _, o_h, _, _, _ = rig.oracle()
+    assert_close(out.float().cpu().numpy(), o_out, TOL["bf16"], "node outputs")
+    assert_close(rig.states()[0], o_h, TOL_STATE, "node SSM states")
+
+
 def test_node_order_within_a_level_changes_no_bit():
     cfg = parity.small_config(1536, "bf16")
     rig = ProjRig(cfg, gen.random_branching_tree(32, 5, 2), 48)
@@ -147,7 +180,7 @@ def test_matches_the_split_mode_calls():
 
 def test_bad_slot_is_reported_and_skipped():
     cfg = parity.small_config(256, "f32")
-    rig = ProjRig(cfg, gen.full_tree([2]), 8)
+    rig = ProjRig(cfg, gen.full_tree([2]), 8, nodes_per_cluster=2)
     rig.node_slot[2] = rig.cache.n_slots + 3
     rig.step(np.arange(1))
     assert int(rig.status.item()) == 0
