@@ -1,5 +1,5 @@
 """Seeded random sweep of the prefill over shapes, modes, chunk plans, block widths and slot arrangements, and of the
-tree step over random trees, each case against the fp64 oracle.  The cases are small (the oracle takes milliseconds)
+tree step (plain and with the projections inside) over random trees, each case against the fp64 oracle.  The cases are small (the oracle takes milliseconds)
 but cross every tile, chunk and block boundary in many different ways."""
 
 import numpy as np
@@ -132,3 +132,46 @@ def test_random_tree_case(seed):
         assert_close(cache.ssm[0, 1:].cpu().numpy(), o_h, TOL_STATE, "node states")
     if mode != "preconv":
         assert np.array_equal(cache.conv[0, 1:].float().cpu().numpy().astype(np.float64), o_conv)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_projection_tree_case(seed):
+    """Random width (every block width and cluster size, ragged last blocks), rank, tree, grouping, dtype, A and step-size mode."""
+    g = np.random.default_rng(900 + seed)
+    act = "bf16" if g.random() < 0.6 else "f32"
+    Dn = int(g.choice([8, 72, 128, 136, 392, 520, 1024, 1032, 1536, 2048, 2056, 3072, 4096]))
+    R = int(g.choice([8, 16, 24, 48, 64, 96, 160, 256]))
+    n_levels = int(g.integers(1, 5))
+    n_nodes = min(int(g.integers(n_levels, 4 * n_levels + 1)), 1 + 4 * (n_levels - 1))
+    tree = gen.random_branching_tree(n_nodes, n_levels, seed, max_children=4) if n_levels > 1 else gen.chain_tree(1)
+    cfg = parity.small_config(Dn, act, cid=93, seed=seed)
+    general_A = bool(g.random() < 0.5)
+    params = gen.layer_params(cfg, 0, conv_bias=bool(g.random() < 0.5), general_A=general_A)
+    flags = md.MDRAFT_DT_SOFTPLUS | (md.MDRAFT_A_POWERS if (not general_A and g.random() < 0.7) else 0)
+    W_x, W_dt = gen.select_proj(cfg, 0, R)
+    tdt = torch_act(act)
+    M = tree.n_nodes
+    x, z, _, _, _ = gen.node_inputs(cfg, 0, 0, M)
+    have_root_state = bool(g.random() < 0.7)
+    h0 = g.normal(size=(Dn, 16)).astype(np.float32)
+    c0 = gen.round_to_act(g.normal(size=(3, Dn)).astype(np.float32), act)
+    cache = md.StateCache(1, 1 + M, Dn, act=tdt)
+    cache.ssm[0, 0] = torch.from_numpy(h0).cuda()
+    cache.conv[0, 0] = to_device(c0, tdt)
+    parent_slot = np.where(tree.parents < 0, 0 if have_root_state else -1, tree.parents + 1).astype(np.int32)
+    node_slot = (np.arange(M) + 1).astype(np.int32)
+    lay = upload_layer(params, act, flags)
+    dx, dz, dWx, dWdt = (to_device(a, tdt) for a in (x, z, W_x, W_dt))
+    out = torch.full((M, Dn), float("nan"), dtype=tdt, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    npc = int(g.choice([0, 1, 2, 4]))
+    for lo, hi in zip(tree.level_offsets[:-1], tree.level_offsets[1:]):
+        md.mdraft_tree_step_proj(lay, cache, 0, dWx, dWdt, dx[lo:hi], dz[lo:hi], out[lo:hi], i32(parent_slot[lo:hi]), i32(node_slot[lo:hi]),
+                                 status, nodes_per_cluster=npc)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    olay = oracle.layer_from_params(params, parity.oracle_flags(flags))
+    o_out, o_conv, o_h, _, _, _ = oracle.tree_proj(olay, W_x, W_dt, tree.parents, x, z, c0 if have_root_state else None, h0 if have_root_state else None)
+    assert_close(out.float().cpu().numpy(), o_out, TOL[act], "node outputs")
+    assert_close(cache.ssm[0, 1:].cpu().numpy(), o_h, TOL_STATE, "node states")
+    assert np.array_equal(cache.conv[0, 1:].float().cpu().numpy().astype(np.float64), o_conv)
