@@ -577,7 +577,9 @@ def run_ours(args):
         while total < 10.0 and reps < 64:   # whole steps of the oracle until about 10 s of work are on the clock
             _, dt, used = time_oracle_sample(w, NL, cores)
             total += dt; reps += 1
+        v1, dt1, _ = time_oracle_sample(w, 2, 1)   # the same oracle on one thread, two layers of the step
         cpu = {"value": reps * units_step / total, "unit": UNIT, "cores": used, "kind": "oracle", "seconds": total,
+               "single_thread": {"value": v1, "unit": UNIT, "seconds": dt1, "sample": "2 of the 24 layers of one step, one thread"},
                "sample": "%d repetitions of the whole step (24 layers: prefill 2048 tokens + 150-node tree path by path + commit), fp64" % reps}
 
     if rank == 0:
