@@ -350,11 +350,27 @@ __global__ void __launch_bounds__(CB) tree_proj_kernel(const TreeProjArgs p) {
     cluster_wait();
     {
         const uint32_t nblk = cluster_size();
-        for (int idx = tid; idx < NT * rows; idx += CB) {
-            const int i = idx / rows, r = idx - i * rows;
-            float sum = 0.f;
-            for (uint32_t c = 0; c < nblk; ++c) sum += peer_block_float(&s_part[i * kMaxRows + r], c);
-            s_s[i * kMaxRows + r] = sum;
+        if constexpr (NT == 1) {
+            // Narrow level, latency counts: all remote reads of an entry are in flight together; the additions keep
+            // the blocks' order.
+            for (int r = tid; r < rows; r += CB) {
+                float part[kProjMaxCluster];
+#pragma unroll
+                for (int c = 0; c < kProjMaxCluster; ++c) part[c] = (uint32_t)c < nblk ? peer_block_float(&s_part[r], c) : 0.f;
+                float sum = 0.f;
+#pragma unroll
+                for (int c = 0; c < kProjMaxCluster; ++c)
+                    if ((uint32_t)c < nblk) sum += part[c];
+                s_s[r] = sum;
+            }
+        } else {
+            // Wide level: the registers are better spent elsewhere (measured), other blocks cover the waits.
+            for (int idx = tid; idx < NT * rows; idx += CB) {
+                const int i = idx / rows, r = idx - i * rows;
+                float sum = 0.f;
+                for (uint32_t c = 0; c < nblk; ++c) sum += peer_block_float(&s_part[i * kMaxRows + r], c);
+                s_s[i * kMaxRows + r] = sum;
+            }
         }
     }
     cluster_arrive();  // this block no longer reads its neighbours; the matching wait is the last thing it does
