@@ -566,6 +566,17 @@ def run_ours(args):
                     torch.cuda.synchronize()
                     ts.append((time.perf_counter() - t0) * 1e3)
                 drafter[mode][name] = statistics.median(ts)
+                if fused:   # the same round as one replayed graph (one host launch per round)
+                    for _ in range(3):
+                        td.draft_round_one_graph(11, cfg_t)
+                    torch.cuda.synchronize()
+                    ts = []
+                    for _ in range(10):
+                        t0 = time.perf_counter()
+                        td.draft_round_one_graph(11, cfg_t)
+                        torch.cuda.synchronize()
+                        ts.append((time.perf_counter() - t0) * 1e3)
+                    drafter.setdefault("projection_step_one_graph_per_round", {})[name] = statistics.median(ts)
             if int(td.status.item()):
                 raise RuntimeError("device status bits set in the drafter leg")
             del td

@@ -61,6 +61,8 @@ class ToyDrafter:
         self.y = torch.zeros((max_nodes, d_inner), dtype=act, device=device)
         self.logits = torch.zeros((max_nodes, vocab), dtype=act, device=device)
         self._graphs = {}
+        self._round_graphs = {}
+        self.root_token = torch.zeros(1, dtype=torch.int64, device=device)   # read by the round, so that a captured round can be replayed with another root
 
     @staticmethod
     def _norm(h: torch.Tensor) -> torch.Tensor:
@@ -106,14 +108,13 @@ class ToyDrafter:
             self._graphs[key] = g
         g.replay()
 
-    def draft_round(self, root_token: int, config: Sequence[int], use_graph: bool = True):
-        """Draft one tree below the committed state.  config = (N_1, ..., N_gamma) as the paper writes it; the root
-        (the last verified token) is node 0.  Returns (tokens (M,), parents list); node states are in slots 1..M."""
+    def _round(self, config: Sequence[int], use_graph: bool):
+        """All generations of one draft tree below the committed state, root token taken from `self.root_token`."""
         parents = [-1]
         level = [0]
-        self.tokens[0] = root_token
-        self.parent_slot[0] = 0
-        self.node_slot[0] = 1
+        self.tokens[0:1] = self.root_token
+        self.parent_slot[0:1] = 0
+        self.node_slot[0:1] = 1
         self.generation(0, 1, use_graph)
         lo = 1
         for n_i in config:
@@ -128,6 +129,31 @@ class ToyDrafter:
             level = list(range(lo, lo + width))
             lo += width
         return self.tokens[:lo].clone(), parents
+
+    def draft_round(self, root_token: int, config: Sequence[int], use_graph: bool = True):
+        """Draft one tree below the committed state.  config = (N_1, ..., N_gamma) as the paper writes it; the root
+        (the last verified token) is node 0.  Returns (tokens (M,), parents list); node states are in slots 1..M.
+        With `use_graph` every generation step is one replayed CUDA graph; the host launches them and the top-k
+        between them."""
+        self.root_token.fill_(int(root_token))
+        return self._round(config, use_graph)
+
+    def draft_round_one_graph(self, root_token: int, config: Sequence[int]):
+        """The same round as ONE replayed CUDA graph per tree configuration (the paper's graph cache, Section 4.1, taken
+        to the whole round: generation steps, top-k and index bookkeeping all sit inside the graph, so the host does one
+        launch per round).  Returns (tokens (M,), parents list); the token tensor is overwritten by the next replay."""
+        key = tuple(int(v) for v in config)
+        self.root_token.fill_(int(root_token))
+        entry = self._round_graphs.get(key)
+        if entry is None:
+            self._round(key, use_graph=False)   # first use of every shape happens outside the capture
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                out = self._round(key, use_graph=False)
+            entry = self._round_graphs[key] = (g, out)
+        entry[0].replay()
+        return entry[1]
 
     def commit(self, node: int) -> None:
         mb.mdraft_state_commit(self.cache, torch.tensor([1 + node], dtype=torch.int32, device=self.dev),

@@ -71,3 +71,19 @@ def test_toy_drafter_tree_matches_path_replica(fused):
     d.commit(4)
     torch.cuda.synchronize()
     assert torch.equal(d.cache.ssm[:, 0], d.cache.ssm[:, 5]) and torch.equal(d.cache.conv[:, 0], d.cache.conv[:, 5])
+
+
+def test_whole_round_in_one_graph_equals_generation_by_generation():
+    d = ToyDrafter(n_layers=2, d_model=32, d_inner=64, dt_rank=8, vocab=97, max_nodes=32, act=torch.float32, seed=3, fused=True)
+    g = torch.Generator(device="cuda").manual_seed(4)
+    d.cache.ssm[:, 0] = torch.randn(d.cache.ssm[:, 0].shape, generator=g, device="cuda")
+    d.cache.conv[:, 0] = torch.randn(d.cache.conv[:, 0].shape, generator=g, device="cuda")
+    for root in (5, 41, 5):   # the second and third calls replay the captured round with another root token
+        tok_a, par_a = d.draft_round(root, (3, 2, 1), use_graph=False)
+        logits_a = d.logits[:len(par_a)].clone()
+        states_a = d.cache.ssm[:, 1:1 + len(par_a)].clone()
+        tok_b, par_b = d.draft_round_one_graph(root, (3, 2, 1))
+        torch.cuda.synchronize()
+        assert int(d.status.item()) == 0
+        assert par_a == par_b and torch.equal(tok_a, tok_b)
+        assert torch.equal(logits_a, d.logits[:len(par_a)]) and torch.equal(states_a, d.cache.ssm[:, 1:1 + len(par_a)])
