@@ -645,16 +645,18 @@ __global__ void __launch_bounds__(kCarryGroups * 32) carry_kernel(const PrefillA
     float4 a2 = __ldg(reinterpret_cast<const float4*>(p.L.A + (size_t)dd * kN) + quad);
     a2.x *= kLog2e; a2.y *= kLog2e; a2.z *= kLog2e; a2.w *= kLog2e;
     grid_release_dependents();
-    grid_wait();  // the summaries are the work of the kernel just before
-
+    // Sequence offsets, slots and the starting state are inputs of the call: the summary pass ahead of this kernel
+    // let it start only after everything before the call had finished, so they may be read before the wait below.
     int first, nck;
     seq_chunks(p.cu, p.n_seq, p.T, p.chunk_len, s, first, nck);
-    if (nck <= 1) return;
     const int islot = load_slot(p.init_slot, s), fslot = load_slot(p.final_slot, s);
-    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;  // the output pass reports it
-
+    const bool slots_ok = islot < p.pool.n_slots && fslot < p.pool.n_slots;
     float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (islot >= 0) carry = *(reinterpret_cast<const float4*>(p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)dd * kN) + quad);
+    if (nck > 1 && slots_ok && islot >= 0)
+        carry = *(reinterpret_cast<const float4*>(p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)dd * kN) + quad);
+    grid_wait();  // the summaries are the work of the kernel just before
+    if (nck <= 1) return;
+    if (!slots_ok) return;  // the output pass reports it
     const size_t per_chunk = (size_t)D * (kN / 4);  // float4s in one chunk's [N/4][D] block
     const size_t col = (size_t)quad * D + dd;        // this thread's float4 inside such a block
     float4* wsq = reinterpret_cast<float4*>(p.ws_q);
