@@ -203,6 +203,12 @@ def test_argument_checks():
     assert e.value.status == -2
     with pytest.raises(ValueError):
         md.mdraft_tree_step_proj(rig.lay, rig.cache, 0, rig.dW_dt, rig.dW_x, *one)
+    with pytest.raises(md.MdraftError) as e:
+        md.mdraft_tree_step_proj(rig.lay, rig.cache, 0, rig.dW_x, rig.dW_dt, *one, nodes_per_cluster=3)
+    assert e.value.status == -1
+    with pytest.raises(md.MdraftError) as e:   # weights must start on a 16-byte boundary
+        md.mdraft_tree_step_proj(rig.lay, rig.cache, 0, torch.zeros(40 * 256 + 1, dtype=rig.tdt, device="cuda")[1:].view(40, 256), rig.dW_dt, *one)
+    assert e.value.status == -3
     wide = parity.small_config(4104, "bf16")
     lay = upload_layer(gen.layer_params(wide, 0), "bf16", md.MDRAFT_DT_SOFTPLUS)
     cache = md.StateCache(1, 2, 4104, act=rig.tdt)
