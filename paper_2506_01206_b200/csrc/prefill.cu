@@ -347,7 +347,7 @@ __device__ __forceinline__ void issue_tile(unsigned char* stage, uint64_t* bar, 
 
 // ---------------------------------------------------------------------------------------------------
 template <typename AT, int SUB, bool kPow, bool kOut, bool kFast>
-__global__ void __launch_bounds__(SUB * kBoxCols + 32) chunk_kernel(const PrefillArgs p, const __grid_constant__ PrefillMaps maps) {
+__global__ void __launch_bounds__(SUB * kBoxCols + 32, SUB == 1 ? 4 : 1) chunk_kernel(const PrefillArgs p, const __grid_constant__ PrefillMaps maps) {
     constexpr int TT = TileTokens<AT>::v;
     constexpr int kCB = SUB * kBoxCols;          // channels per block, one thread each
     constexpr int kStageBytes = stage_bytes(SUB);
