@@ -8,8 +8,13 @@
 // them to the child's slot with bulk stores.  Forking therefore costs one read and one write of the state and
 // no copy pass, all traffic is in multi-KB contiguous pieces, and the bytes in flight do not depend on how many
 // registers a thread holds.  Siblings are separate blocks that re-read the parent (the second reader finds it in
-// L2), so a level's latency does not grow with its branching factor.  The wait on the mbarrier is bounded: if it
+// L2), so a level's latency does not grow with its branching factor.  The waits on the mbarriers are bounded: if one
 // runs out the block raises MDRAFT_DEV_WAIT_EXPIRED, waits once more (bounded) for its copies, and returns.
+//
+// The levels of one call follow one another through programmatic dependent launch: a level's blocks start while the
+// level before is still running, look up their slots, fetch the layer constants (and, from the third level of a call on, the node's
+// input rows), and only then wait for the kernel ahead, after which the parent's state and window are fetched.  Every
+// block passes that wait on every path, so a level's completion implies the completion of everything before it.
 #include "common.cuh"
 #include "tree_step.cuh"
 
@@ -18,7 +23,8 @@ namespace mdraft {
 namespace {
 
 constexpr int kTB = kTreeThreads;            // channels per block
-constexpr uint32_t kSpinLimit = 1u << 20;    // polls of the mbarrier before the block gives up
+constexpr uint32_t kSpinLimit = 1u << 20;
+    // polls of the mbarrier before the block gives up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -54,7 +60,7 @@ __device__ __forceinline__ void xor_permute(float4 (&t)[4], int sw) {
 }
 
 template <typename AT, bool kPow>
-__global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p) {
+__global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p, const int early_inputs, const int ordinary_launch) {
     __shared__ __align__(128) float4 s_h[kTB * (kN / 4)];  // state slice [channel][quad]
     __shared__ __align__(16) AT s_conv[kW - 1][kTB];
     __shared__ __align__(16) AT s_x[kTB];                 // the node's x row; receives the out row afterwards
@@ -62,8 +68,12 @@ __global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p) {
     __shared__ __align__(16) AT s_dt[kTB];
     __shared__ __align__(16) AT s_B[kN];
     __shared__ __align__(16) AT s_C[kN];
-    __shared__ __align__(8) uint64_t bar;
+    __shared__ __align__(8) uint64_t bar, bar_in;
 
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the next level may begin its own look-ups
+    // Launched the ordinary way nothing runs ahead of this kernel: the wait costs nothing, and passing it first lets
+    // every copy be requested at once.
+    if (ordinary_launch) asm volatile("griddepcontrol.wait;" ::: "memory");
     const int D = p.L.d_inner;
     const int node = p.lvl_begin + blockIdx.x;
     const int tid = threadIdx.x;
@@ -75,6 +85,7 @@ __global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p) {
     const int nslot = __ldg(p.node_slot + node);
     if (pslot < -1 || pslot >= p.pool.n_slots || nslot < 0 || nslot >= p.pool.n_slots) {  // the node becomes a no-op
         if (tid == 0 && blockIdx.y == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         return;
     }
     const uint32_t flags = p.L.flags;
@@ -86,23 +97,35 @@ __global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p) {
     AT* conv_parent = static_cast<AT*>(p.pool.conv) + (size_t)pslot * p.pool.conv_slot_stride + d0;
     AT* conv_child = static_cast<AT*>(p.pool.conv) + (size_t)nslot * p.pool.conv_slot_stride + d0;
 
-    if (tid == 0) {
-        mbar_init(&bar, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // Inputs of the node (x, z, dt, B, C rows) go on one mbarrier, the parent's state and window on another: the
+    // former may be requested before the kernel ahead has finished when the caller says they cannot be its work.
+    auto issue_inputs = [&]() {
         uint32_t total = row_bytes;
-        if (!conv_only) total += 2 * row_bytes + 2 * bc_bytes + (have_parent ? h_bytes : 0u);
+        if (!conv_only) total += 2 * row_bytes + 2 * bc_bytes;
+        mbar_expect_tx(&bar_in, total);
+        bulk_load(s_x, static_cast<const AT*>(p.x) + (size_t)node * p.ldx + d0, row_bytes, &bar_in);
+        if (!conv_only) {
+            bulk_load(s_z, static_cast<const AT*>(p.z) + (size_t)node * p.ldz + d0, row_bytes, &bar_in);
+            bulk_load(s_dt, static_cast<const AT*>(p.dt) + (size_t)node * p.lddt + d0, row_bytes, &bar_in);
+            bulk_load(s_B, static_cast<const AT*>(p.B) + (size_t)node * p.ldb, bc_bytes, &bar_in);
+            bulk_load(s_C, static_cast<const AT*>(p.C) + (size_t)node * p.ldc, bc_bytes, &bar_in);
+        }
+    };
+    auto issue_state = [&]() {
+        uint32_t total = 0;
+        if (!conv_only && have_parent) total += h_bytes;
         if (!preconv && have_parent) total += (kW - 1) * row_bytes;
         mbar_expect_tx(&bar, total);
-        bulk_load(s_x, static_cast<const AT*>(p.x) + (size_t)node * p.ldx + d0, row_bytes, &bar);
-        if (!conv_only) {
-            if (have_parent) bulk_load(s_h, h_parent, h_bytes, &bar);
-            bulk_load(s_z, static_cast<const AT*>(p.z) + (size_t)node * p.ldz + d0, row_bytes, &bar);
-            bulk_load(s_dt, static_cast<const AT*>(p.dt) + (size_t)node * p.lddt + d0, row_bytes, &bar);
-            bulk_load(s_B, static_cast<const AT*>(p.B) + (size_t)node * p.ldb, bc_bytes, &bar);
-            bulk_load(s_C, static_cast<const AT*>(p.C) + (size_t)node * p.ldc, bc_bytes, &bar);
-        }
+        if (!conv_only && have_parent) bulk_load(s_h, h_parent, h_bytes, &bar);
         if (!preconv && have_parent)
             for (int j = 0; j < kW - 1; ++j) bulk_load(s_conv[j], conv_parent + (size_t)j * D, row_bytes, &bar);
+    };
+    if (tid == 0) {
+        mbar_init(&bar, 1);
+        mbar_init(&bar_in, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (early_inputs || ordinary_launch) issue_inputs();
+        if (ordinary_launch) issue_state();
     }
 
     // Layer constants travel by ordinary loads while the copies are in flight.
@@ -128,12 +151,19 @@ __global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p) {
             dsk = p.L.D ? __ldg(p.L.D + d) : 0.f;
         }
     }
-    __syncthreads();  // the mbarrier is initialised for everyone
-    const bool ok = mbar_wait_bounded(&bar, 0u);
+    if (!ordinary_launch) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // everything read from here on may be the work of the kernel ahead
+        if (tid == 0) {
+            if (!early_inputs) issue_inputs();
+            issue_state();
+        }
+    }
+    __syncthreads();  // the mbarriers are initialised for everyone
+    const bool ok = mbar_wait_bounded(&bar_in, 0u) && mbar_wait_bounded(&bar, 0u);
     if (__syncthreads_or(!ok)) {
         if (tid == 0) {
             flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
-            mbar_wait_bounded(&bar, 0u);  // the copies target this block's shared memory: give them one more bounded chance
+            mbar_wait_bounded(&bar_in, 0u); mbar_wait_bounded(&bar, 0u);
         }
         return;
     }
@@ -217,19 +247,40 @@ __global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p) {
 
 }  // namespace
 
+// The first level of a call is launched the ordinary way: what runs ahead of it is usually somebody else's kernel (a
+// projection), which never releases its dependents early, and behind such a kernel a programmatic launch was measured
+// 0.8 us slower than an ordinary one.  Later levels follow a level of the same call and are launched programmatically.
+template <typename K>
+cudaError_t launch_level(K kernel, dim3 grid, cudaStream_t st, const TreeArgs& p, int early) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kTB);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.level_in_call > 0 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, p, early, p.level_in_call > 0 ? 0 : 1);
+}
+
 cudaError_t launch_tree_step(const TreeArgs& p, int act, cudaStream_t st) {
     const int n = p.lvl_end - p.lvl_begin;
     if (n <= 0) return cudaSuccess;
     const bool pow = p.L.flags & MDRAFT_A_POWERS;
+    // From the third level of a call on, the two kernels that may still be running when this one starts are levels of
+    // the same call, which write states and `out` rows of other nodes only: the node's input rows cannot be their work
+    // and are requested before the wait.  The first two levels follow kernels of unknown origin and request nothing
+    // but slot indices and layer constants early.
+    const int early = p.level_in_call >= 2 ? 1 : 0;
     dim3 grid(n, (p.L.d_inner + kTB - 1) / kTB);
     if (act == MDRAFT_F32) {
-        if (pow) tree_step_kernel<float, true><<<grid, kTB, 0, st>>>(p);
-        else tree_step_kernel<float, false><<<grid, kTB, 0, st>>>(p);
-    } else {
-        if (pow) tree_step_kernel<__nv_bfloat16, true><<<grid, kTB, 0, st>>>(p);
-        else tree_step_kernel<__nv_bfloat16, false><<<grid, kTB, 0, st>>>(p);
+        if (pow) return launch_level(tree_step_kernel<float, true>, grid, st, p, early);
+        return launch_level(tree_step_kernel<float, false>, grid, st, p, early);
     }
-    return cudaGetLastError();
+    if (pow) return launch_level(tree_step_kernel<__nv_bfloat16, true>, grid, st, p, early);
+    return launch_level(tree_step_kernel<__nv_bfloat16, false>, grid, st, p, early);
 }
 
 }  // namespace mdraft
