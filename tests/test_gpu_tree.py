@@ -237,3 +237,48 @@ def test_round_graph_cache_replays_what_eager_launches_compute():
         assert torch.equal(graph_stack.cache.conv.view(torch.int16), eager_stack.cache.conv.view(torch.int16))
     assert replayed == [False, False, True] and len(cache) == 2
     graph_stack.check_status(); eager_stack.check_status()
+
+
+@pytest.mark.parametrize("act", ["f32", "bf16"])
+def test_chained_launches_keep_their_order_when_buffers_are_shared(act):
+    """Levels of one call start while the level ahead still runs.  Two arrangements in which a late read would show:
+    (a) `out` is the same buffer as `x` (every node overwrites its own input row), all levels in one call;
+    (b) a conv-only call whose output is the very next call's pre-convolved input, nothing in between.
+    Both, replayed many times from one CUDA graph, must give the bits of the level-by-level run."""
+    cfg = parity.small_config(392, act)
+    tree = gen.paper_tree((3, 2, 2, 1, 1))
+    rig = TreeRig(cfg, tree)
+    ref = rig.run_levels()
+    h_ref, c_ref = rig.states()
+    lv = [int(v) for v in tree.level_offsets]
+    par, nod = i32(rig.parent_slot), i32(rig.node_slot)
+    x0 = rig.dev[0].clone()
+    xio = rig.dev[0].clone()
+    u = torch.empty_like(x0); y = torch.empty_like(x0)
+
+    def in_place():
+        xio.copy_(x0)
+        md.mdraft_tree_step(rig.lay, rig.cache, 0, xio, rig.dev[1], rig.dev[2], rig.dev[3], rig.dev[4], xio, par, nod, lv, rig.status)
+
+    def split():
+        md.mdraft_tree_step(rig.lay, rig.cache, 0, x0, None, None, None, None, u, par, nod, lv, rig.status, flags=md.MDRAFT_CONV_ONLY)
+        md.mdraft_tree_step(rig.lay, rig.cache, 0, u, rig.dev[1], rig.dev[2], rig.dev[3], rig.dev[4], y, par, nod, lv, rig.status,
+                            flags=md.MDRAFT_DT_SOFTPLUS | md.MDRAFT_PRECONV)
+
+    for fn, result in ((in_place, xio), (split, y)):
+        rig.reset()
+        fn(); torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        for _ in range(20):
+            rig.reset()
+            g.replay()
+        torch.cuda.synchronize()
+        assert int(rig.status.item()) == 0
+        h, c = rig.states()
+        if fn is in_place:
+            assert torch.equal(result, ref) and np.array_equal(h, h_ref) and np.array_equal(c, c_ref)
+        else:   # split mode rounds u to the activation dtype on the way: equal within tolerance, states likewise
+            assert_close(result.float().cpu().numpy(), ref.float().cpu().numpy(), 3 * TOL[act], "split-mode chain")
+            assert_close(h, h_ref, 3 * TOL[act], "split-mode chain states")
