@@ -290,11 +290,14 @@ int mdraft_tree_step(const mdraft_layer* layer, const mdraft_cache* cache, int32
     a.ldx = ldx; a.ldz = ldz; a.lddt = lddt; a.ldb = ldb; a.ldc = ldc; a.ldo = ldo;
     a.parent_slot = parent_slot; a.node_slot = node_slot; a.dev_status = dev_status;
     const int levels = level_offsets ? n_levels : 1;
+    int launched = 0;  // an empty level launches nothing and must not count: the chaining rules go by kernels ahead
     for (int l = 0; l < levels; ++l) {
-        a.level_in_call = l;
+        a.level_in_call = launched;
         a.lvl_begin = level_offsets ? level_offsets[l] : 0;
         a.lvl_end = level_offsets ? level_offsets[l + 1] : n_nodes;
+        if (a.lvl_end == a.lvl_begin) continue;
         if (launch_tree_step(a, act, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MDRAFT_ERR_CUDA;
+        ++launched;
     }
     return MDRAFT_OK;
 }

@@ -14,7 +14,7 @@ struct TreeArgs {
     void* out;
     int64_t ldx, ldz, lddt, ldb, ldc, ldo;
     const int32_t *parent_slot, *node_slot;
-    int level_in_call;       // 0 for the first level launched by a call
+    int level_in_call;       // kernels this call has launched before this level (0 for the first)
     int lvl_begin, lvl_end;  // nodes [lvl_begin, lvl_end) form one tree level
     int32_t* dev_status;
 };
