@@ -78,9 +78,9 @@ struct PrefillPlan {
 
 // Chunk length: split the token axis until every SM holds kBlocksPerSm blocks of kPrefillThreads channels (one
 // resident wave, no tail), but never into chunks shorter than kMinChunk tokens (per-chunk set-up would dominate).
-// When one wave would need chunks longer than kOneWaveMax tokens (long or batched contexts), several waves of short
-// chunks do better: blocks are then handed out as SMs free up, which evens out uneven sequences and keeps every SM
-// busy to the end (measured: 32768 tokens 404 -> 367 us, 32 packed sequences of 1k-8k tokens 1607 -> 1512 us).
+// When one wave would need chunks longer than kOneWaveMax tokens and the chunks would be uneven (packed batches) or the
+// blocks narrow, several waves of short chunks do better: blocks are then handed out as SMs free up, which evens out
+// uneven sequences and keeps every SM busy to the end (32 packed sequences of 1k-8k tokens: 1607 -> 1512 us).
 constexpr int kBlocksPerSm = 4, kMinChunk = 32, kOneWaveMax = 256, kManyWavesChunk = 128, kManyWavesChunkBatched = 256;
 
 PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen, const mdraft_prefill_opts* opts) {
@@ -102,7 +102,11 @@ PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen
         if (want < 1) want = 1;
         Lc = (T + want - 1) / want;
         if (Lc < kMinChunk) Lc = kMinChunk;
-        if (Lc > kOneWaveMax) {  // several waves: narrow blocks, four to an SM, so that a new block's set-up hides behind the others
+        // A single sequence in wide blocks stays in one wave at any length: 49 x 3 equal chunks finish together
+        // (32768 tokens: 344 us against 372-376 for several waves of short chunks; 65536: 675 against 724).  Packed
+        // batches, whose sequences differ in length, and widths that do not fill wide blocks take several waves of
+        // short chunks in narrow blocks, four to an SM, so that a new block's set-up hides behind the others.
+        if (Lc > kOneWaveMax && !(wide && n_seq == 1)) {
             Lc = n_seq > 1 ? kManyWavesChunkBatched : kManyWavesChunk;
             if (forced == 0) wide = false;
         }
