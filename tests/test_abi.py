@@ -117,3 +117,33 @@ def test_missing_library_is_a_loud_error(tmp_path):
     from paper_2506_01206_b200 import binding
     with pytest.raises(ImportError):
         binding.load_library(str(tmp_path / "nope.so"))
+
+
+def test_projection_step_host_side_checks(lib):
+    """mdraft_tree_step_proj turns bad arguments away before any launch (so this runs without a GPU)."""
+    from paper_2506_01206_b200 import binding
+    INVALID, UNSUPPORTED, MISALIGNED = -1, -2, -3
+    layer, cache = _layer(binding), _cache(binding)
+
+    def call(layer=layer, cache=cache, W_x=0x900000, W_dt=0xA00000, rank=8, npc=0, x=0x100000, z=0x200000, out=0x600000, n=1,
+             par=0x700000, nod=0x800000, ldx=64):
+        pr = binding._SelectProj(W_x, W_dt, rank, npc)
+        return lib.mdraft_tree_step_proj(C.byref(layer), C.byref(cache), 0, C.byref(pr) if W_x is not None else None, x, ldx, z, 64, out, 64,
+                                         n, par, nod, None, None)
+
+    assert call(rank=12) == UNSUPPORTED            # not a multiple of 8
+    assert call(rank=264) == UNSUPPORTED           # beyond the shared-memory vectors
+    assert call(rank=0) == UNSUPPORTED
+    big = _cache(binding, ssm_slot_stride=4104 * 16, ssm_layer_stride=4 * 4104 * 16, conv_slot_stride=3 * 4104, conv_layer_stride=12 * 4104)
+    assert call(layer=_layer(binding, d_inner=4104), cache=big, ldx=4104) == UNSUPPORTED   # more than one cluster of the widest blocks
+    assert call(layer=_layer(binding, flags=1 | 2)) == INVALID           # pre-convolved input makes no sense here
+    assert call(layer=_layer(binding, flags=1 | 4)) == INVALID
+    assert call(W_x=None) == INVALID
+    assert call(W_dt=0) == INVALID
+    assert call(W_x=0x900008) == MISALIGNED
+    assert call(npc=3) == INVALID
+    assert call(n=-1) == INVALID
+    assert call(x=None) == INVALID
+    assert call(ldx=32) == INVALID
+    assert call(par=None) == INVALID
+    assert call(n=0, par=None, nod=None) == 0      # nothing to do is not an error
