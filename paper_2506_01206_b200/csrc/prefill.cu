@@ -44,6 +44,7 @@ __host__ __device__ constexpr int off_z(int sub) { return 2 * sub * kTileBytes; 
 __host__ __device__ constexpr int off_b(int sub) { return 3 * sub * kTileBytes; }
 __host__ __device__ constexpr int off_c(int sub) { return 3 * sub * kTileBytes + kBCBytes; }
 __host__ __device__ constexpr int smem_bytes(int sub) { return kStages * (stage_bytes(sub) + 2 * kBCBytes * 2); }  // + fp32 B, C
+constexpr int kFmaPairs = 1;            // pairs of decays per token computed on the FMA pipe when A is general (measured: 0 -> 43.8, 1 -> 42.5, 2 -> 43.0, 3 -> 45.6 us per 2048x1536 call)
 constexpr int GRP = 4;                  // tokens whose state-independent part is computed together (measured: 2 % faster than one by one)
 constexpr uint32_t kSpinLimit = 1u << 20;  // polls of one mbarrier before the block gives up
 
@@ -72,6 +73,39 @@ __device__ __forceinline__ u64 mul2(u64 a, u64 b) {
     u64 d;
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
+}
+
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+    u64 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// 2^x for a pair of arguments x <= 0 on the FMA pipe instead of the special-function unit (which a general A keeps
+// busy with 16 exponentials per token, channel and pass).  x = j + f with j = round(x) taken from the mantissa of
+// x + 1.5*2^23 and f in [-0.5, 0.5]; 2^f = 1 + f g(f) with g of degree 4 interpolated at Chebyshev nodes (relative error
+// 2.8e-7 at most, 1e-8 on average: the accuracy of ex2.approx, and exactly 1 at 0); the result's exponent field then takes j.  Arguments below -126 are raised to -126
+// (the true value is below 1.2e-38 there and the product with the state flushes to zero either way).
+__device__ __forceinline__ u64 exp2_pair_fma(u64 x) {
+    float lo, hi;
+    unpk(x, lo, hi);
+    x = pk(fmaxf(lo, -126.0f), fmaxf(hi, -126.0f));
+    const u64 magic = pk(12582912.0f, 12582912.0f);
+    const u64 t = add2(x, magic);                                   // integer part in the low mantissa bits
+    const u64 r = add2(t, pk(-12582912.0f, -12582912.0f));          // round(x) as a float
+    const u64 f = fma2(r, pk(-1.0f, -1.0f), x);                     // x - round(x)
+    u64 q = pk(0.0013381302f, 0.0013381302f);                      // (2^f - 1) / f ...
+    q = fma2(q, f, pk(0.009666368f, 0.009666368f));
+    q = fma2(q, f, pk(0.05550381f, 0.05550381f));
+    q = fma2(q, f, pk(0.2402235f, 0.2402235f));
+    q = fma2(q, f, pk(0.6931472f, 0.6931472f));
+    q = fma2(q, f, pk(1.0f, 1.0f));                                 // ... so that 2^0 is exactly 1
+    float qlo, qhi, tlo, thi;
+    unpk(q, qlo, qhi);
+    unpk(t, tlo, thi);
+    qlo = __int_as_float(__float_as_int(qlo) + (__float_as_int(tlo) << 23));
+    qhi = __int_as_float(__float_as_int(qhi) + (__float_as_int(thi) << 23));
+    return pk(qlo, qhi);
 }
 
 // ---------------------------------------------------------------- mbarrier + bulk copy
@@ -252,11 +286,18 @@ struct ChannelScan {
             for (int k = 0; k < 4; ++k) P[4 + k] = mul2(P[k], R8);
         } else {
             const u64 dd = pk(delta, delta);
+            // With a step size known to be >= 0 (softplus) the arguments are <= 0 and the last kFmaPairs pairs go to
+            // the FMA pipe, which takes a little load off the special-function unit.
+            constexpr int kMufuPairs = kFast ? kN / 2 - kFmaPairs : kN / 2;
 #pragma unroll
             for (int k = 0; k < kN / 2; ++k) {
-                float lo, hi;
-                unpk(mul2(dd, a2[k]), lo, hi);
-                P[k] = pk(ex2(lo), ex2(hi));
+                if (k < kMufuPairs) {
+                    float lo, hi;
+                    unpk(mul2(dd, a2[k]), lo, hi);
+                    P[k] = pk(ex2(lo), ex2(hi));
+                } else {
+                    P[k] = exp2_pair_fma(mul2(dd, a2[k]));
+                }
             }
         }
     }
