@@ -147,3 +147,21 @@ def test_projection_step_host_side_checks(lib):
     assert call(ldx=32) == INVALID
     assert call(par=None) == INVALID
     assert call(n=0, par=None, nod=None) == 0      # nothing to do is not an error
+
+
+def test_prefill_plan_seen_through_the_workspace_query(lib):
+    """The chunk plan is host logic; its workspace query shows it: one wave of equal chunks for a single sequence at
+    any length (so the scratch stops growing with the context), several waves of short chunks for a packed batch."""
+    from paper_2506_01206_b200 import binding
+    layer = _layer(binding, d_inner=1536, act=1)
+    q = lambda T, S, mx, opts=None: lib.mdraft_prefill_workspace_bytes(C.byref(layer), T, S, mx, opts)
+    per_chunk = 1536 * 16 * 4 + 1536 * 4          # one summary: state + summed step size
+    assert q(8, 1, 8) == 0                         # shorter than one chunk: nothing to carry
+    one = [q(T, 1, T) for T in (2048, 8192, 32768, 131072)]
+    assert all(b > 0 for b in one)
+    assert max(one) <= 52 * per_chunk + 4 * per_chunk, "a single sequence stays at about 49 chunks whatever its length"
+    packed = q(141650, 32, 8192)
+    assert packed > 10 * max(one), "a packed batch is cut into many short chunks"
+    o = binding._PrefillOpts(chunk_len=64, block_channels=0)
+    assert q(2048, 1, 2048, C.byref(o)) >= 32 * per_chunk      # a forced chunk length is honoured
+    assert q(0, 1, 8) == 0 and q(8, 0, 8) == 0     # nonsense sizes give 0, not garbage
