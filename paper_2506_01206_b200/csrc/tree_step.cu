@@ -12,9 +12,10 @@
 // runs out the block raises MDRAFT_DEV_WAIT_EXPIRED, waits once more (bounded) for its copies, and returns.
 //
 // The levels of one call follow one another through programmatic dependent launch: a level's blocks start while the
-// level before is still running, look up their slots, fetch the layer constants (and, from the third level of a call on, the node's
-// input rows), and only then wait for the kernel ahead, after which the parent's state and window are fetched.  Every
-// block passes that wait on every path, so a level's completion implies the completion of everything before it.
+// level before is still running, look up their slots, fetch the layer constants (and, from the third level of a call
+// on, the node's input rows), and only then wait for the kernel ahead, after which the parent's state and window are
+// fetched.  Every block passes that wait on every path, so a level's completion implies the completion of everything
+// before it.
 #include "common.cuh"
 #include "tree_step.cuh"
 
@@ -23,8 +24,7 @@ namespace mdraft {
 namespace {
 
 constexpr int kTB = kTreeThreads;            // channels per block
-constexpr uint32_t kSpinLimit = 1u << 20;
-    // polls of the mbarrier before the block gives up
+constexpr uint32_t kSpinLimit = 1u << 20;    // polls of an mbarrier before the block gives up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kTB) tree_step_kernel(const TreeArgs p, const 
     AT* conv_child = static_cast<AT*>(p.pool.conv) + (size_t)nslot * p.pool.conv_slot_stride + d0;
 
     // Inputs of the node (x, z, dt, B, C rows) go on one mbarrier, the parent's state and window on another: the
-    // former may be requested before the kernel ahead has finished when the caller says they cannot be its work.
+    // former may be requested before the kernel ahead has finished when the launch says they cannot be its work.
     auto issue_inputs = [&]() {
         uint32_t total = row_bytes;
         if (!conv_only) total += 2 * row_bytes + 2 * bc_bytes;
