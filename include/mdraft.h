@@ -200,7 +200,10 @@ int mdraft_conv_scan_prefill_noalloc(const mdraft_layer *layer, const mdraft_cac
  *                   Level l = nodes [level_offsets[l], level_offsets[l+1]); levels are launched in
  *                   order on `stream`, so a parent may live in an earlier level of the same call.
  * Hazards (caller's duty): within one level no node_slot may equal another node's parent_slot or
- * node_slot; parent_slot[i] == node_slot[i] (in-place chain decode) is fine.  The result of a node
+ * node_slot; parent_slot[i] == node_slot[i] (in-place chain decode) is fine.  Within one call the
+ * input rows of a node (x, z, dt, B, C) must not be rows that another node of the same call writes
+ * (`out` may be the same buffer as `x` as long as node i writes row i only): the levels of a call
+ * overlap their set-up, and a level may fetch its input rows before the levels ahead have finished.  The result of a node
  * does not depend on where in the level it sits or on how levels are split across calls.
  */
 int mdraft_tree_step(const mdraft_layer *layer, const mdraft_cache *cache, int32_t layer_index,
