@@ -203,8 +203,9 @@ int mdraft_conv_scan_prefill_noalloc(const mdraft_layer *layer, const mdraft_cac
  * node_slot; parent_slot[i] == node_slot[i] (in-place chain decode) is fine.  Within one call the
  * input rows of a node (x, z, dt, B, C) must not be rows that another node of the same call writes
  * (`out` may be the same buffer as `x` as long as node i writes row i only): the levels of a call
- * overlap their set-up, and a level may fetch its input rows before the levels ahead have finished.  The result of a node
- * does not depend on where in the level it sits or on how levels are split across calls.
+ * overlap their set-up, and a level may fetch its input rows before the levels ahead have finished.
+ * The result of a node does not depend on where in the level it sits or on how levels are split
+ * across calls.
  */
 int mdraft_tree_step(const mdraft_layer *layer, const mdraft_cache *cache, int32_t layer_index,
                      const void *x, int64_t ldx, const void *z, int64_t ldz, const void *dt, int64_t lddt,
