@@ -12,8 +12,8 @@
 // runs out the block raises MDRAFT_DEV_WAIT_EXPIRED, waits once more (bounded) for its copies, and returns.
 //
 // The levels of one call follow one another through programmatic dependent launch: a level's blocks start while the
-// level before is still running, look up their slots, fetch the layer constants (and, from the third level of a call
-// on, the node's input rows), and only then wait for the kernel ahead, after which the parent's state and window are
+// level before is still running, look up their slots, fetch the layer constants and the node's input
+// rows, and only then wait for the kernel ahead, after which the parent's state and window are
 // fetched.  Every block passes that wait on every path, so a level's completion implies the completion of everything
 // before it.
 #include "common.cuh"
@@ -269,11 +269,11 @@ cudaError_t launch_tree_step(const TreeArgs& p, int act, cudaStream_t st) {
     const int n = p.lvl_end - p.lvl_begin;
     if (n <= 0) return cudaSuccess;
     const bool pow = p.L.flags & MDRAFT_A_POWERS;
-    // From the third level of a call on, the two kernels that may still be running when this one starts are levels of
-    // the same call, which write states and `out` rows of other nodes only: the node's input rows cannot be their work
-    // and are requested before the wait.  The first two levels follow kernels of unknown origin and request nothing
-    // but slot indices and layer constants early.
-    const int early = p.level_in_call >= 2 ? 1 : 0;
+    // The first kernel of a call is an ordinary launch: it starts only after everything ahead of the call has finished.
+    // A later level starts when the level before it does, so the only kernels that can still be running then are
+    // levels of this call, which write states and `out` rows of other nodes only: the node's input rows cannot be
+    // their work and are requested before the wait.
+    const int early = p.level_in_call >= 1 ? 1 : 0;
     dim3 grid(n, (p.L.d_inner + kTB - 1) / kTB);
     if (act == MDRAFT_F32) {
         if (pow) return launch_level(tree_step_kernel<float, true>, grid, st, p, early);
