@@ -3,8 +3,11 @@
  *
  * C ABI.  Plain pointers and sizes only; no C++ or framework types.  Unless a
  * parameter says HOST, every pointer is a DEVICE pointer owned by the caller;
- * the library allocates nothing, keeps no pointer after a call returns, and has
- * no global state.  All work is enqueued on `stream` (a cudaStream_t passed as
+ * the library allocates nothing and keeps no caller pointer after a call
+ * returns.  Its only state between calls is the fixed scratch array of
+ * mdraft_conv_scan_prefill_noalloc and that array's cached per-device address
+ * (see the sharing rules at its declaration); every other entry point is
+ * stateless.  All work is enqueued on `stream` (a cudaStream_t passed as
  * void*; NULL = the default stream) and no entry point synchronises with the
  * host, except where stated.
  *

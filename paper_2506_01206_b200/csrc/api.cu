@@ -1,4 +1,5 @@
-// C ABI of the library: argument checks, launch planning, dispatch.  No allocation, no global state.
+// C ABI of the library: argument checks, launch planning, dispatch.  Nothing here allocates or keeps state between
+// calls (the one exception in the library is the fixed scratch array of mdraft_conv_scan_prefill_noalloc, noalloc.cu).
 #include <cudaTypedefs.h>
 #include <limits.h>
 
@@ -191,7 +192,8 @@ int mdraft_version(void) { return 100; }
 size_t mdraft_prefill_workspace_bytes(const mdraft_layer* layer, int32_t total_tokens, int32_t n_seq, int32_t max_seqlen,
                                       const mdraft_prefill_opts* opts) {
     if (check_layer(layer) != MDRAFT_OK || total_tokens <= 0 || n_seq <= 0 || max_seqlen <= 0) return 0;
-    return plan_prefill(layer, total_tokens, n_seq, max_seqlen, opts).bytes;
+    // No sequence is longer than the whole batch: a looser static bound must not change the plan.
+    return plan_prefill(layer, total_tokens, n_seq, max_seqlen < total_tokens ? max_seqlen : total_tokens, opts).bytes;
 }
 
 int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cache, int32_t layer_index,
@@ -226,9 +228,13 @@ int mdraft_conv_scan_prefill(const mdraft_layer* layer, const mdraft_cache* cach
     if ((rc = check_matrix(dt, lddt, D, act, have_rows && !conv_only))) return rc;
     if ((rc = check_matrix(B, ldb, kN, act, have_rows && !conv_only))) return rc;
     if ((rc = check_matrix(C, ldc, kN, act, have_rows && !conv_only))) return rc;
+    // The same bound as in the workspace query: no sequence is longer than the whole batch.  A batch of empty
+    // sequences therefore never takes the chunked path (and needs no workspace), whatever static bound was given.
+    const int plan_tokens = total_tokens > 0 ? total_tokens : 1;
+    if (max_seqlen > plan_tokens) max_seqlen = plan_tokens;
     if (max_seqlen < 1) max_seqlen = 1;
 
-    PrefillPlan pl = plan_prefill(layer, total_tokens > 0 ? total_tokens : 1, n_seq, max_seqlen, opts);
+    PrefillPlan pl = plan_prefill(layer, plan_tokens, n_seq, max_seqlen, opts);
     if (pl.chunked) {
         if (!workspace || workspace_bytes < pl.bytes) return MDRAFT_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MDRAFT_ERR_MISALIGNED;

@@ -14,6 +14,21 @@ constexpr int kW = 4;             // d_conv handled by these kernels
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
+// Every wait on an mbarrier polls at most this often before the block gives up, raises MDRAFT_DEV_WAIT_EXPIRED
+// and returns.  One poll is a try_wait that may suspend the thread for at most kPollNs nanoseconds (a stated limit
+// instead of the system's own), so a wait that never completes ends after about a second.  The two macros exist for the failure-path tests only: a second build of the library with a short
+// limit and with every copy barrier told to expect a few bytes more than will ever arrive, so that each bounded
+// wait runs out (the copies themselves still land) and the give-up paths execute on a healthy GPU.
+#ifndef MDRAFT_SPIN_LIMIT
+#define MDRAFT_SPIN_LIMIT (1u << 20)
+#endif
+#ifndef MDRAFT_TEST_OVERSTATE_TX
+#define MDRAFT_TEST_OVERSTATE_TX 0u
+#endif
+constexpr uint32_t kSpinLimit = MDRAFT_SPIN_LIMIT;
+constexpr uint32_t kOverstateTx = MDRAFT_TEST_OVERSTATE_TX;
+constexpr uint32_t kPollNs = 1000u;
+
 // ---------------------------------------------------------------- scalar math
 __device__ __forceinline__ float ex2(float v) {
     float r;

@@ -46,7 +46,6 @@ __host__ __device__ constexpr int off_c(int sub) { return 3 * sub * kTileBytes +
 __host__ __device__ constexpr int smem_bytes(int sub) { return kStages * (stage_bytes(sub) + 2 * kBCBytes * 2); }  // + fp32 B, C
 constexpr int kFmaPairs = 1;            // pairs of decays per token computed on the FMA pipe when A is general (measured: 0 -> 43.8, 1 -> 42.5, 2 -> 43.0, 3 -> 45.6 us per 2048x1536 call)
 constexpr int GRP = 4;                  // tokens whose state-independent part is computed together (measured: 2 % faster than one by one)
-constexpr uint32_t kSpinLimit = 1u << 20;  // polls of one mbarrier before the block gives up
 
 template <typename AT> struct TileTokens { static constexpr int v = kPrefillTileRowBytes / (int)sizeof(AT); };  // 16 (bf16) or 8 (fp32)
 
@@ -115,7 +114,7 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes + kOverstateTx) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -123,9 +122,9 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kPollNs)
         : "memory");
     return ok != 0;
 }

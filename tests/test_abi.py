@@ -89,6 +89,13 @@ def test_host_side_argument_checks(lib):
     assert _prefill(lib, binding, ok_layer, ok_cache, opts=C.byref(bad)) == INVALID
     # nothing to do is fine and launches nothing
     assert _prefill(lib, binding, ok_layer, ok_cache, n_seq=0, T=0, cu=None) == 0
+    # A batch of empty sequences needs no workspace whatever static length bound comes with it: the query says 0 and
+    # the call must agree (it may only fail later, at the launch, where there is no GPU).
+    assert lib.mdraft_prefill_workspace_bytes(C.byref(ok_layer), 0, 2, 5000, None) == 0
+    assert _prefill(lib, binding, ok_layer, ok_cache, T=0, n_seq=2, max_seqlen=5000, x=None, z=None, dt=None, B=None, C=None, out=None,
+                    final=0x800000) != WORKSPACE
+    # and a static bound looser than the batch itself does not change the plan
+    assert lib.mdraft_prefill_workspace_bytes(C.byref(ok_layer), 8, 1, 100000, C.byref(opts)) == need
 
     def tree(layer=ok_layer, cache=ok_cache, n=4, parent=0xA00000, node=0xB00000, n_levels=1, levels=None, x=0x100000):
         return lib.mdraft_tree_step(C.byref(layer), C.byref(cache) if cache is not None else None, 0, x, 64, 0x200000, 64,

@@ -210,3 +210,29 @@ def test_prefill_flags_bad_sequence_lengths_and_slots():
     torch.cuda.synchronize()
     assert int(status.item()) & md.MDRAFT_DEV_BAD_SLOT
     assert float(out[:10].abs().max()) > 0 and float(out[10:].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("act", ["f32", "bf16"])
+def test_batch_of_empty_sequences_moves_the_state_and_needs_no_workspace(act):
+    """No tokens at all: every sequence's final state is its starting state, copied from slot to slot (zeros where
+    there is no starting slot), with no workspace even when the caller's static length bound is large."""
+    Dn, S = 136, 3
+    tdt = torch.float32 if act == "f32" else torch.bfloat16
+    cfg = parity.small_config(Dn, act, S)
+    prob = parity.make_problem(cfg, [4])   # only for the layer constants
+    lay = upload_layer(prob.params, act, md.MDRAFT_DT_SOFTPLUS)
+    assert md.mdraft_prefill_workspace_bytes(lay, 0, S, 5000) == 0
+    cache = md.StateCache(1, 2 * S, Dn, act=tdt)
+    cache.ssm.normal_(); cache.conv.normal_()
+    before_h, before_c = cache.ssm.clone(), cache.conv.clone()
+    empty = torch.empty((0, Dn), dtype=tdt, device="cuda")
+    empty_bc = torch.empty((0, 16), dtype=tdt, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    init = i32([0, -1, 2]); final = i32([3, 4, 2])
+    md.mdraft_conv_scan_prefill(lay, cache, 0, empty, empty, empty, empty_bc, empty_bc, empty, i32([0, 0, 0, 0]), 5000, init, final, None, 0, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(cache.ssm[0, 3], before_h[0, 0]) and torch.equal(cache.conv[0, 3], before_c[0, 0])
+    assert float(cache.ssm[0, 4].abs().max()) == 0.0 and float(cache.conv[0, 4].float().abs().max()) == 0.0
+    for s in (0, 1, 2, 5):
+        assert torch.equal(cache.ssm[0, s], before_h[0, s]) and torch.equal(cache.conv[0, s], before_c[0, s])

@@ -2,8 +2,8 @@
 
 It exists for callers that must not allocate on the device while they run (a server whose memory pool is
 fixed at start-up, a plug-in that is handed pointers but owns no allocator).  The check is simple: on the same
-inputs it must give what the ordinary entry point gives with a caller-owned workspace, and it must keep doing
-so when called again, because every call reuses the one scratch array and finds the previous call's leftovers
+inputs it must give, bit for bit, what the ordinary entry point gives with a caller-owned workspace (and that must
+agree with the fp64 oracle), and it must keep doing so when called again, because every call reuses the one scratch array and finds the previous call's leftovers
 in it.  This file sorts last on purpose, so that a run which stops at the first failure has already run every
 other test; it also passes when run alone in a fresh process.
 """
@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import parity
 from parity import TOL, TOL_STATE, assert_close
 
@@ -34,7 +35,8 @@ def test_noalloc_prefill_equals_prefill_with_workspace_twice(act):
     lens = [300, 41, 222]
     S, T, Dn, chunk = len(lens), sum(lens), 264, 32
     cfg = parity.small_config(Dn, act, S)
-    lay, tdt, dev = _device_problem(parity.make_problem(cfg, lens, conv_bias=True, general_A=True))
+    prob = parity.make_problem(cfg, lens, conv_bias=True, general_A=True)
+    lay, tdt, dev = _device_problem(prob)
     cu = i32(np.concatenate([[0], np.cumsum(lens)]))
     final = i32(np.arange(S))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -54,10 +56,16 @@ def test_noalloc_prefill_equals_prefill_with_workspace_twice(act):
         md.mdraft_conv_scan_prefill_noalloc(lay, cache_b, 0, *dev, out_b, cu, max(lens), None, final, chunk, status)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
-        assert_close(out_b.float().cpu().numpy(), out_a.float().cpu().numpy(), TOL[act], f"call {call}: out")
-        assert_close(cache_b.ssm.cpu().numpy(), cache_a.ssm.cpu().numpy(), TOL_STATE, f"call {call}: SSM state")
-        assert torch.equal(cache_b.conv.view(torch.int16 if act == "bf16" else torch.int32),
-                           cache_a.conv.view(torch.int16 if act == "bf16" else torch.int32)), f"call {call}: conv window"
+        # the same kernels on the same plan, only the scratch lives elsewhere: the same bits
+        bits = torch.int16 if act == "bf16" else torch.int32
+        assert torch.equal(out_b.view(bits), out_a.view(bits)), f"call {call}: out"
+        assert torch.equal(cache_b.ssm.view(torch.int32), cache_a.ssm.view(torch.int32)), f"call {call}: SSM state"
+        assert torch.equal(cache_b.conv.view(bits), cache_a.conv.view(bits)), f"call {call}: conv window"
+        # and the right ones: against the fp64 oracle, at the tolerances of the parity tests
+        o_out, o_conv, o_h = oracle.prefill(oracle.layer_from_params(prob.params), prob.x, prob.z, prob.dt, prob.B, prob.C, prob.cu)
+        assert_close(out_b.float().cpu().numpy(), o_out, TOL[act], f"call {call}: out against the oracle")
+        assert_close(cache_b.ssm[0].cpu().numpy(), o_h, TOL_STATE, f"call {call}: SSM state against the oracle")
+        assert np.array_equal(cache_b.conv[0].float().cpu().numpy().astype(np.float64), o_conv), f"call {call}: conv window against the oracle"
 
 
 def test_noalloc_prefill_refuses_problems_beyond_its_scratch():
