@@ -9,6 +9,7 @@ workload (Mamba-130M: 24 layers, d_inner 1536, d_state 16; context 2048 tokens; 
 the per-phase throughputs (prefill token*channels/s, tree node-updates/s) are reported beside it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py --profile-case prefill|tree|proj [sizes ...]     (small runs of one kernel family for a profiler)
 
 N > 1 (under torchrun) runs N independent replicas (the path has no exchange step): weak scaling.
 `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
@@ -187,10 +188,19 @@ def run_reference(args):
 # 16 states x (form the decay, decay*h, input*B, C*h) 64 + skip 1 + gate 4
 ALU_LANE_OPS_PER_UNIT = 82
 FP32_LANES_PER_SM, SM_COUNT, SM_MAX_MHZ = 128, 148, 1965.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/ (set to None
-# whenever the kernel changes after the counters were taken)
-NCU_TRAFFIC_OUTPUT_PASS = 24.01e6   # chunk_kernel<bf16, structured A, output pass>, 2048 x 1536
-NCU_TRAFFIC_TREE_WIDEST = 32.54e6   # tree_step_kernel<bf16>, 442-node level of the 32 x 32-node round
+def ncu_traffic(key):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the named kernel, from the ncu capture recorded in
+    profiles/traffic.json, or None when a source file of that kernel has changed since the capture (the record keeps
+    the SHA-256 of the sources it was taken with, so a stale figure cannot be reported by accident)."""
+    import hashlib
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))[key]
+        for rel, digest in rec["sources_sha256"].items():
+            if hashlib.sha256(open(os.path.join(ROOT, rel), "rb").read()).hexdigest() != digest:
+                return None, rec.get("kernel")
+        return float(rec["dram_bytes_per_launch"]), rec.get("kernel")
+    except Exception:
+        return None, None
 
 
 class BatchedTree:
@@ -419,6 +429,51 @@ def run_ours(args):
                   "plain_step_inputs_given": time_graph(capture(pj_plain), Kp, 3) / NL * 1e3}
     if int(bt_status.item()):
         raise RuntimeError("device status bits set in the projection leg")
+
+    # ---- further prefill shapes (time per layer-call, CUDA-graph replay over distinct per-layer buffers that together
+    # exceed L2): the long context, the packed batch and fp32 activations.  These legs time only; their inputs are drawn
+    # on the device from the recipe's distributions (x, z, B, C ~ N(0,1), dt = clip(0.5 N(0,1))), the parity of these
+    # shapes against the oracle is the business of tests/test_gpu_configs.py.
+    def prefill_leg(act, lens, n_buf, reps):
+        tdt_l = torch_act(act)
+        es = 4 if act == "f32" else 2
+        S_l, T_l = len(lens), int(sum(lens))
+        gen_t = torch.Generator(device=dev); gen_t.manual_seed(1234 + rank)
+        def rnd(shape, scale=1.0):
+            return (torch.randn(shape, generator=gen_t, device=dev, dtype=torch.float32) * scale).to(tdt_l)
+        bufs = []
+        for _ in range(n_buf):
+            dtv = rnd((T_l, D), 0.5).float().clamp_(float(gen.DT_PRE_LO), float(gen.DT_PRE_HI)).to(tdt_l)
+            bufs.append([rnd((T_l, D)), rnd((T_l, D)), dtv, rnd((T_l, 16)), rnd((T_l, 16))])
+        outs_l = [torch.empty((T_l, D), dtype=tdt_l, device=dev) for _ in range(n_buf)]
+        lays = [upload_layer(w.params[l], act, md.MDRAFT_DT_SOFTPLUS | (md.MDRAFT_A_POWERS if is_pow else 0), dev) for l in range(n_buf)]
+        st_l = DrafterStack(lays, S_l, T_l, S_l, max(lens), 0, dev)
+        cu_l = None if S_l == 1 else i32(np.concatenate([[0], np.cumsum(lens)]), dev)
+        slots_l = i32(np.arange(S_l), dev)
+        fn = lambda: st_l.prefill(bufs, outs_l, cu_l, max(lens), None, slots_l)
+        ms = time_graph(capture(fn), reps, 3) / n_buf
+        st_l.check_status()
+        bytes_l = 4 * es * T_l * D + 2 * 16 * es * T_l + S_l * (D * 16 * 4 + 3 * D * es)
+        units = T_l * D
+        del bufs, outs_l, st_l
+        torch.cuda.empty_cache()
+        return {"activations": act, "sequences": S_l, "tokens": T_l, "us_per_layer": ms * 1e3, "token_channels_per_s": units / (ms * 1e-3),
+                "algorithmic_bytes_per_layer": bytes_l, "hbm_frac": bytes_l / (ms * 1e-3) / 1e9 / load_peaks()[0],
+                "fp32_issue_frac_82_ops": ALU_LANE_OPS_PER_UNIT * units / (ms * 1e-3) / (SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6),
+                "fp32_issue_frac_70_ops": 70 * units / (ms * 1e-3) / (SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6),
+                "buffers": n_buf, "launches_per_layer": 3}
+
+    prefill_shapes = None
+    if not args.quick:
+        cfg4_lens = [int(v) for v in np.diff(gen.seq_lengths(gen.get_config(4)))]
+        prefill_shapes = {
+            "note": "whole prefill call (summary pass + carry scan + output pass) per layer; hbm_frac against the measured copy bandwidth; "
+                    "fp32_issue_frac = lane-operations per token*channel (82 as counted in DESIGN.md, 70 as the scope table estimated) x units / time / (148 x 128 x 1965 MHz)",
+            "long_context_32768_bf16": prefill_leg("bf16", [32768], 4, 5),
+            "packed_batch_32_seqs_1k_8k_bf16": prefill_leg("bf16", cfg4_lens, 2, 3),
+            "fp32_activations_2048": prefill_leg("f32", [2048], 8, 10),
+            "bf16_activations_2048_device_inputs": prefill_leg("bf16", [2048], 8, 10),
+        }
     clocks = sampler.stop()
 
     # ---- end to end: pinned host inputs -> device -> the path -> outputs back to the host, every step, through the
@@ -502,7 +557,7 @@ def run_ours(args):
         # the bound that applies is the fp32 issue rate; the HBM figure is kept beside it.
         "bound": "alu", "kernel": kname, "achieved": lane_ops / scan_s / 1e12, "peak": alu_peak / 1e12,
         "unit": "T fp32 lane-op/s (one instruction on one lane; an FMA counts once)", "frac": lane_ops / scan_s / alu_peak,
-        "traffic": NCU_TRAFFIC_OUTPUT_PASS,
+        "traffic": ncu_traffic("prefill_output_pass")[0], "traffic_kernel": ncu_traffic("prefill_output_pass")[1],
         "peak_source": "148 SMs x 128 fp32 lanes x %.0f MHz (clocks.max.sm)" % SM_MAX_MHZ,
         "algorithmic_lane_ops_per_launch": lane_ops, "algorithmic_bytes_per_launch": pb, "launch_us": output_pass_us,
         "timed": "CUDA-graph replay of 24 launches of this kernel alone (the 2048 rows as 49 unsplit sequences of 42 tokens: same grid, block and tokens per block as in the chunked call), time / 24",
@@ -520,7 +575,7 @@ def run_ours(args):
     roofline_tree = {
         "bound": "hbm", "kernel": "tree_step_kernel<bf16>", "workload": "32 sequences x 32-node trees, widest level (%d nodes), 24 layers" % (hi - lo),
         "achieved": NL * bt_wide_bytes / (ms_bt_widest * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
-        "frac": NL * bt_wide_bytes / (ms_bt_widest * 1e-3) / 1e9 / peak, "traffic": NCU_TRAFFIC_TREE_WIDEST,
+        "frac": NL * bt_wide_bytes / (ms_bt_widest * 1e-3) / 1e9 / peak, "traffic": ncu_traffic("tree_step_widest_level")[0], "traffic_kernel": ncu_traffic("tree_step_widest_level")[1],
         "algorithmic_bytes_per_launch": bt_wide_bytes, "launch_us": 1e3 * ms_bt_widest / NL,
         "timed": "CUDA-graph replay of 24 launches (one per layer, distinct 110 MB pools), time / 24",
         "whole_round": {"ms": ms_bt_round, "levels": [b - a for a, b in zip(bt.levels[:-1], bt.levels[1:])],
@@ -613,12 +668,76 @@ def run_ours(args):
             "roofline_tree_step": roofline_tree,
             "phases": extra,
             "general_A": general,
+            "prefill_shapes": prefill_shapes,
             "projection_level": proj_level,
             "drafter_round": drafter,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     replicas.finish(world)
+
+
+# ----------------------------------------------------------------------------------------------- profiler cases
+def profile_case(what, sizes):
+    """Small, self-contained runs of one kernel family for a profiler (ncu): few launches, well under 1 GB on the device,
+    inputs larger than L2 across the layers so that DRAM counters still mean something.
+      prefill [tokens=2048] [layers=4] [reps=3] [fp32=0]   130M-shaped context encode, bf16 (or fp32) activations, structured A
+      tree    [layers=4] [reps=2]                          one batched-serving draft round, 32 sequences x 32-node trees
+      proj    [nodes=18] [layers=24] [reps=3]              one tree level through the step that forms dt, B, C itself"""
+    import torch
+    import paper_2506_01206_b200 as md
+    from paper_2506_01206_b200.device_inputs import i32, to_device, torch_act, upload_layer
+    flags = md.MDRAFT_DT_SOFTPLUS | md.MDRAFT_A_POWERS
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if what == "prefill":
+        tokens, n_layers, reps, fp32 = (list(sizes) + [2048, 4, 3, 0][len(sizes):])[:4]
+        cfg = gen.get_config(1)
+        act = "f32" if fp32 else cfg.act
+        tdt, D = torch_act(act), cfg.d_inner
+        lays = [upload_layer(gen.layer_params(cfg, l), act, flags) for l in range(n_layers)]
+        ins = [[to_device(a, tdt) for a in gen.prefill_inputs(cfg, l, tokens)] for l in range(n_layers)]
+        outs = [torch.empty((tokens, D), dtype=tdt, device="cuda") for _ in range(n_layers)]
+        cache = md.StateCache(n_layers, 1, D, act=tdt)
+        ws = torch.empty(max(256, md.mdraft_prefill_workspace_bytes(lays[0], tokens, 1, tokens)), dtype=torch.uint8, device="cuda")
+        slot = i32([0])
+        for _ in range(reps):
+            for l in range(n_layers):
+                md.mdraft_conv_scan_prefill(lays[l], cache, l, *ins[l], outs[l], None, tokens, None, slot, ws, 0, status)
+        torch.cuda.synchronize()
+        print("prefill: %d tokens x %d channels, %s, %d layers x %d, status %d" % (tokens, D, act, n_layers, reps, int(status.item())))
+    elif what == "tree":
+        n_layers, reps = (list(sizes) + [4, 2][len(sizes):])[:2]
+        bt = BatchedTree(seed=0)
+        cfg, D = bt.cfg, bt.cfg.d_inner
+        tdt = torch_act(cfg.act)
+        lays = [upload_layer(gen.layer_params(cfg, l), cfg.act, flags) for l in range(n_layers)]
+        ins = [[to_device(a, tdt) for a in gen.node_inputs(cfg, l, 0, bt.M)] for l in range(n_layers)]
+        outs = [torch.empty((bt.M, D), dtype=tdt, device="cuda") for _ in range(n_layers)]
+        cache = md.StateCache(n_layers, bt.S + bt.M, D, act=tdt)
+        cache.ssm.normal_()
+        par, nod = i32(bt.parent), i32(bt.nodes)
+        for _ in range(reps):
+            for l in range(n_layers):
+                md.mdraft_tree_step(lays[l], cache, l, *ins[l], outs[l], par, nod, bt.levels, status)
+        torch.cuda.synchronize()
+        print("tree: %d nodes, levels %s, %d layers x %d, status %d" % (bt.M, np.diff(bt.levels).tolist(), n_layers, reps, int(status.item())))
+    else:
+        n_nodes, n_layers, reps = (list(sizes) + [18, 24, 3][len(sizes):])[:3]
+        dt_rank = 48
+        cfg = gen.get_config(1)
+        tdt, D = torch_act(cfg.act), cfg.d_inner
+        lays = [upload_layer(gen.layer_params(cfg, l), cfg.act, flags) for l in range(n_layers)]
+        Ws = [[to_device(v, tdt) for v in gen.select_proj(cfg, l, dt_rank)] for l in range(n_layers)]
+        ins = [[to_device(a, tdt) for a in gen.node_inputs(cfg, l, 0, n_nodes)[:2]] for l in range(n_layers)]
+        out = torch.empty((n_nodes, D), dtype=tdt, device="cuda")
+        cache = md.StateCache(n_layers, 1 + n_nodes, D, act=tdt)
+        cache.ssm.normal_(); cache.conv.normal_()
+        par, nod = i32([0] * n_nodes), i32(list(range(1, n_nodes + 1)))
+        for _ in range(reps):
+            for l in range(n_layers):
+                md.mdraft_tree_step_proj(lays[l], cache, l, Ws[l][0], Ws[l][1], ins[l][0], ins[l][1], out, par, nod, status)
+        torch.cuda.synchronize()
+        print("proj: %d nodes x %d channels, dt_rank %d, %d layers x %d, status %d" % (n_nodes, D, dt_rank, n_layers, reps, int(status.item())))
 
 
 def main():
@@ -628,8 +747,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--quick", action="store_true", help="skip the further prefill shapes (long context, packed batch, fp32)")
+    ap.add_argument("--profile-case", choices=["prefill", "tree", "proj"], help="run one small kernel case for a profiler and exit")
+    ap.add_argument("sizes", nargs="*", type=int, help="sizes of the profile case (see profile_case)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile_case:
+        profile_case(args.profile_case, args.sizes)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
