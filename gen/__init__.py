@@ -25,6 +25,9 @@ from .draw import (
     DT_BIAS,
     DT_PRE_LO,
     DT_PRE_HI,
+    SsdParams,
+    ssd_params,
+    ssd_inputs,
 )
 from .trees import (
     Tree,
@@ -40,7 +43,7 @@ from .trees import (
 __all__ = [
     "CONFIGS", "Config", "get_config", "LayerParams", "layer_params",
     "prefill_inputs", "node_inputs", "seq_lengths", "round_to_act",
-    "bf16_bits", "from_bf16_bits", "DT_BIAS", "DT_PRE_LO", "DT_PRE_HI",
+    "bf16_bits", "from_bf16_bits", "DT_BIAS", "DT_PRE_LO", "DT_PRE_HI", "SsdParams", "ssd_params", "ssd_inputs",
     "Tree", "full_tree", "paper_tree", "capped_tree",
     "random_branching_tree", "chain_tree", "random_accepted_node",
     "config_tree",

@@ -141,3 +141,49 @@ def seq_lengths(cfg: Config, seed: Optional[int] = None) -> np.ndarray:
     cu = np.zeros(cfg.n_seq + 1, dtype=np.int32)
     cu[1:] = np.cumsum(lens)
     return cu
+
+
+# ---------------------------------------------------------------- Mamba-2 (SSD) shapes
+@dataclass
+class SsdParams:
+    A: np.ndarray                 # (H,)   float32, <= 0: one scalar per head
+    D: np.ndarray                 # (D,)   float32 skip weight
+    conv_w: np.ndarray            # (D, W) float32
+    conv_b: Optional[np.ndarray]  # (D,)   float32 or None
+    dt_bias: np.ndarray           # (H,)   float32
+    headdim: int
+    d_state: int
+
+
+def ssd_params(cfg: Config, layer: int, headdim: int, d_state: int, seed: Optional[int] = None, *, conv_bias: bool = False) -> SsdParams:
+    """Constants of one SSD layer: A[j] = -(1 + 15 j / (H - 1)) spreads the heads over the same range -(1..16) as the
+    S4D-real rows of the S6 recipe; D = 1; conv taps ~ N(0, 0.5^2); the recipe's step-size bias."""
+    seed = cfg.seed if seed is None else seed
+    Dn, W = cfg.d_inner, cfg.d_conv
+    H = Dn // headdim
+    A = -(1.0 + 15.0 * np.arange(H, dtype=np.float32) / np.float32(max(H - 1, 1))).astype(np.float32)
+    conv_w = (0.5 * rng_for(seed, cfg.cid, layer, 0, "conv_w").standard_normal((Dn, W), dtype=np.float32)).astype(np.float32)
+    conv_b = None
+    if conv_bias:
+        conv_b = (0.25 * rng_for(seed, cfg.cid, layer, 0, "conv_b").standard_normal(Dn, dtype=np.float32)).astype(np.float32)
+    return SsdParams(A, np.ones(Dn, dtype=np.float32), np.ascontiguousarray(conv_w), conv_b, np.full(H, DT_BIAS, dtype=np.float32), headdim, d_state)
+
+
+def ssd_inputs(cfg: Config, layer: int, rnd: int, phase: int, rows: int, headdim: int, d_state: int, seed: Optional[int] = None):
+    """(x, z, dt, B, C) for ``rows`` tokens or nodes of an SSD layer: x, z (rows, D); dt (rows, H); B, C (rows, N), drawn
+    as in the S6 recipe, with B and C scaled by 1 / sqrt(N / 16) so that C.h keeps the recipe's spread at N = 128."""
+    seed = cfg.seed if seed is None else seed
+    Dn = cfg.d_inner
+    H = Dn // headdim
+
+    def normal(name, shape):
+        return rng_for(seed, cfg.cid, layer, rnd, name, phase).standard_normal(shape, dtype=np.float32)
+
+    x = round_to_act(normal("x", (rows, Dn)), cfg.act)
+    z = round_to_act(normal("z", (rows, Dn)), cfg.act)
+    dt = round_to_act(0.5 * normal("dt", (rows, H)), cfg.act)
+    np.clip(dt, DT_PRE_LO, DT_PRE_HI, out=dt)
+    sc = np.float32(1.0 / np.sqrt(d_state / 16.0))
+    B = round_to_act(sc * normal("B", (rows, d_state)), cfg.act)
+    C = round_to_act(sc * normal("C", (rows, d_state)), cfg.act)
+    return x, z, dt, B, C

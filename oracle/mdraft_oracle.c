@@ -260,3 +260,130 @@ int mdo_tree_proj(const mdo_layer *L, int R, const double *Wx, const double *Wdt
     free(path); free(win); free(h); free(u); free(dt); free(s);
     return 0;
 }
+
+/*
+ * ---------------------------------------------------------------------------------------------------------
+ * Mamba-2 (SSD) drafter: the same path with ONE scalar A per head.
+ *
+ * The paper names Mamba-2 as the drop-in that "directly benefits" the approach (Section 1, the paragraph before
+ * Related Work) and defines nothing about it; the recurrence below is the state-space-duality form of the cited
+ * model, kept as close to the S6 statement above as it goes.  The D channels are split into H = D / P heads of P
+ * channels (d = j * P + p); the step size and A are per HEAD, B and C are shared by all heads (one group):
+ *
+ *     u_t[d]     = SiLU( b_d + sum_k w[d][k] * x[t-(W-1)+k][d] )              (as above, per channel)
+ *     Delta_t[j] = softplus( dt_t[j] + dt_bias[j] )                           (or as given, when the flag is off)
+ *     h_t[d][n]  = exp(Delta_t[j] * A[j]) * h_{t-1}[d][n] + Delta_t[j] * B_t[n] * u_t[d]
+ *     y_t[d]     = sum_n C_t[n] * h_t[d][n] + D[d] * u_t[d]
+ *     out_t[d]   = y_t[d] * SiLU(z_t[d])
+ *
+ * Written out token by token, channel by channel: no chunking, no matrix form.  Pins (tests/pins.py): with every
+ * head's A copied to all N states of its P channels and dt copied to the head's channels this IS mdo_prefill /
+ * mdo_tree (which have their own pins); geometric series and cumulative sum in closed form; head indexing by an
+ * input that differs in one head only.
+ */
+typedef struct {
+    int32_t d_inner, headdim, d_state, d_conv;
+    uint32_t flags;
+    const double *A;       /* (H)  one scalar per head, <= 0 */
+    const double *Dskip;   /* (D) or NULL = 0 */
+    const double *conv_w;  /* (D, W) */
+    const double *conv_b;  /* (D) or NULL = 0 */
+    const double *dt_bias; /* (H) or NULL = 0 */
+} mdo_ssd_layer;
+
+/* One token of one channel of head j = d / P.  dt is the head's pre-activation for this token. */
+static double ssd_channel_token(const mdo_ssd_layer *L, int d, double *win, double *h,
+                                double x, double z, double dt, const double *Bt, const double *Ct)
+{
+    const int N = L->d_state, W = L->d_conv, j = d / L->headdim;
+    double u;
+    if (L->flags & MDO_PRECONV) {
+        u = x;
+    } else {
+        double acc = L->conv_b ? L->conv_b[d] : 0.0;
+        for (int k = 0; k < W - 1; ++k) acc += L->conv_w[(size_t)d * W + k] * win[k];
+        acc += L->conv_w[(size_t)d * W + (W - 1)] * x;
+        for (int k = 0; k + 1 < W - 1; ++k) win[k] = win[k + 1];
+        if (W > 1) win[W - 2] = x;
+        u = mdo_silu(acc);
+    }
+    if (L->flags & MDO_CONV_ONLY) return u;
+    double v = dt + (L->dt_bias ? L->dt_bias[j] : 0.0);
+    double delta = (L->flags & MDO_DT_SOFTPLUS) ? mdo_softplus(v) : v;
+    double decay = exp(delta * L->A[j]);
+    double y = 0.0;
+    for (int n = 0; n < N; ++n) {
+        h[n] = decay * h[n] + delta * Bt[n] * u;
+        y += Ct[n] * h[n];
+    }
+    y += (L->Dskip ? L->Dskip[d] : 0.0) * u;
+    return y * mdo_silu(z);
+}
+
+/*
+ * Context encode, packed sequences as in mdo_prefill.  x, z: (T, D); dt: (T, H); B, C: (T, N).
+ * conv_init (n_seq, W-1, D), h_init (n_seq, D, N) may be NULL; so may conv_final, h_final.
+ */
+void mdo_ssd_prefill(const mdo_ssd_layer *L, int n_seq, const int32_t *cu_seqlens,
+                     const double *x, const double *z, const double *dt,
+                     const double *B, const double *C,
+                     const double *conv_init, const double *h_init,
+                     double *out, double *conv_final, double *h_final)
+{
+    const int D = L->d_inner, N = L->d_state, W = L->d_conv, H = D / L->headdim;
+    for (int s = 0; s < n_seq; ++s) {
+        const int t0 = cu_seqlens[s], t1 = cu_seqlens[s + 1];
+#pragma omp parallel for schedule(static)
+        for (int d = 0; d < D; ++d) {
+            double win[16], h[256];
+            for (int k = 0; k < W - 1; ++k)
+                win[k] = conv_init ? conv_init[((size_t)s * (W - 1) + k) * D + d] : 0.0;
+            for (int n = 0; n < N; ++n)
+                h[n] = h_init ? h_init[((size_t)s * D + d) * N + n] : 0.0;
+            for (int t = t0; t < t1; ++t)
+                out[(size_t)t * D + d] = ssd_channel_token(L, d, win, h, x[(size_t)t * D + d], z[(size_t)t * D + d],
+                                                           dt[(size_t)t * H + d / L->headdim], B + (size_t)t * N, C + (size_t)t * N);
+            if (conv_final)
+                for (int k = 0; k < W - 1; ++k) conv_final[((size_t)s * (W - 1) + k) * D + d] = win[k];
+            if (h_final)
+                for (int n = 0; n < N; ++n) h_final[((size_t)s * D + d) * N + n] = h[n];
+        }
+    }
+}
+
+/*
+ * Tree drafting for one sequence, every node rebuilt along its root-to-node path from the committed state, as in
+ * mdo_tree.  x, z: (M, D); dt: (M, H); B, C: (M, N).  Returns 0, or -1 if a parent index is not an earlier node.
+ */
+int mdo_ssd_tree(const mdo_ssd_layer *L, int M, const int32_t *parent,
+                 const double *x, const double *z, const double *dt,
+                 const double *B, const double *C,
+                 const double *conv0, const double *h0,
+                 double *out, double *conv_nodes, double *h_nodes)
+{
+    const int D = L->d_inner, N = L->d_state, W = L->d_conv, H = D / L->headdim;
+    for (int v = 0; v < M; ++v)
+        if (parent[v] >= v || parent[v] < -1) return -1;
+    int *path = (int *)malloc(sizeof(int) * (size_t)(M > 0 ? M : 1));
+    for (int v = 0; v < M; ++v) {
+        int len = 0;
+        for (int a = v; a >= 0; a = parent[a]) path[len++] = a;
+#pragma omp parallel for schedule(static)
+        for (int d = 0; d < D; ++d) {
+            double win[16], h[256], o = 0.0;
+            for (int k = 0; k < W - 1; ++k) win[k] = conv0 ? conv0[(size_t)k * D + d] : 0.0;
+            for (int n = 0; n < N; ++n) h[n] = h0 ? h0[(size_t)d * N + n] : 0.0;
+            for (int jn = len - 1; jn >= 0; --jn) {
+                const size_t a = (size_t)path[jn];
+                o = ssd_channel_token(L, d, win, h, x[a * D + d], z[a * D + d], dt[a * H + d / L->headdim], B + a * N, C + a * N);
+            }
+            out[(size_t)v * D + d] = o;
+            if (conv_nodes)
+                for (int k = 0; k < W - 1; ++k) conv_nodes[((size_t)v * (W - 1) + k) * D + d] = win[k];
+            if (h_nodes)
+                for (int n = 0; n < N; ++n) h_nodes[((size_t)v * D + d) * N + n] = h[n];
+        }
+    }
+    free(path);
+    return 0;
+}

@@ -402,9 +402,99 @@ def pin_proj_zero_weights(L=None):
         _close(hn[v], np.exp(delta[:, None] * lay.A * (depth[v] + 1)) * h0, what=f"zero W_x: state of node {v}")
 
 
+# ------------------------------------------------------------------ Mamba-2 (SSD): one scalar A per head
+def _ssd_problem(i, H=3, P=2, N=5, W=4, T=19, conv_bias=True):
+    g = _rng(i)
+    Dn = H * P
+    A = -g.uniform(0.3, 4.0, H); Dsk = g.normal(size=Dn); w = g.normal(scale=0.5, size=(Dn, W))
+    cb = g.normal(size=Dn) if conv_bias else None
+    bias = g.normal(size=H) - 3
+    lay = oracle.SsdLayer(A, Dsk, w, cb, bias, P, N, flags=oracle.DT_SOFTPLUS)
+    x = g.normal(size=(T, Dn)); z = g.normal(size=(T, Dn)); dt = g.normal(size=(T, H))
+    B = g.normal(size=(T, N)); Cm = g.normal(size=(T, N))
+    return lay, x, z, dt, B, Cm
+
+
+def _ssd_as_s6(lay):
+    """The S6 layer an SSD layer IS: every head's A copied to the N states of its P channels, its step-size bias to
+    its channels.  (Built here with numpy; nothing of the SSD routine is involved.)"""
+    Dn, H, N, W = lay.dims
+    A6 = np.repeat(lay.A, lay.headdim)[:, None] * np.ones((1, N))
+    bias6 = None if lay.dt_bias is None else np.repeat(lay.dt_bias, lay.headdim)
+    return oracle.Layer(A6, lay.D, lay.conv_w, lay.conv_b, bias6, flags=lay.flags)
+
+
+def pin_ssd_is_s6_with_head_constant_A(L=None):
+    """An SSD layer is an S6 layer whose A is constant over the states and over the channels of a head, and whose step
+    size is shared by the channels of a head: prefill and tree must agree with mdo_prefill / mdo_tree (pinned above)
+    on the expanded constants and the expanded dt, including one-channel heads (P = 1)."""
+    for i, (H, P) in enumerate(((3, 2), (4, 1), (1, 5))):
+        lay, x, z, dt, B, Cm = _ssd_problem(30 + i, H=H, P=P)
+        g = _rng(40 + i)
+        Dn, _, N, W = lay.dims
+        cu = np.array([0, 3, 4, 19], dtype=np.int32)
+        ci = g.normal(size=(3, W - 1, Dn)); hi = g.normal(size=(3, Dn, N))
+        got = oracle.ssd_prefill(lay, x, z, dt, B, Cm, cu_seqlens=cu, conv_init=ci, h_init=hi, _lib_override=L)
+        want = oracle.prefill(_ssd_as_s6(lay), x, z, np.repeat(dt, P, axis=1), B, Cm, cu_seqlens=cu, conv_init=ci, h_init=hi, _lib_override=L)
+        for a, b, nm in zip(got, want, ("out", "window", "state")):
+            _close(a, b, what=f"SSD prefill == S6 prefill on expanded constants (H={H}, P={P}): {nm}")
+        parents = np.array([-1, 0, 0, 1, 1, 2, 4, 4])
+        M = len(parents)
+        got = oracle.ssd_tree(lay, parents, x[:M], z[:M], dt[:M], B[:M], Cm[:M], conv0=ci[0], h0=hi[0], _lib_override=L)
+        want = oracle.tree(_ssd_as_s6(lay), parents, x[:M], z[:M], np.repeat(dt[:M], P, axis=1), B[:M], Cm[:M], conv0=ci[0], h0=hi[0], _lib_override=L)
+        for a, b, nm in zip(got, want, ("out", "window", "state")):
+            _close(a, b, what=f"SSD tree == S6 tree on expanded constants (H={H}, P={P}): {nm}")
+
+
+def pin_ssd_geometric_series(L=None):
+    """Constant Delta, B, C, u per head and a given h0: h_t = a^t h0 + b (1 - a^t) / (1 - a) with the head's scalar
+    a = exp(Delta A), b = Delta B u; A = 0 in one head gives the running sum there."""
+    g = _rng(50)
+    H, P, N, T, W = 3, 2, 4, 33, 4
+    Dn = H * P
+    A = -g.uniform(0.2, 3.0, H); A[1] = 0.0
+    Dsk = g.normal(size=Dn)
+    delta = g.uniform(0.01, 0.3, H)
+    u = g.normal(size=Dn); Bc = g.normal(size=N); Cc = g.normal(size=N)
+    h0 = g.normal(size=(1, Dn, N))
+    lay = oracle.SsdLayer(A, Dsk, _identity_conv(Dn, W), None, None, P, N, flags=oracle.PRECONV)
+    out, _, hT = oracle.ssd_prefill(lay, np.tile(u, (T, 1)), np.full((T, Dn), BIG_Z), np.tile(delta, (T, 1)), np.tile(Bc, (T, 1)), np.tile(Cc, (T, 1)),
+                                    h_init=h0, _lib_override=L)
+    head = np.arange(Dn) // P
+    a = np.exp(delta * A)[head][:, None]                            # (D,1)
+    b = (delta[head] * u)[:, None] * Bc[None, :]                   # (D,N)
+    t = np.arange(1, T + 1)[:, None, None]
+    with np.errstate(invalid="ignore", divide="ignore"):
+        series = np.where(a[None] == 1.0, t * np.ones_like(a)[None], (1 - a[None] ** t) / (1 - a[None]))
+    h = a[None] ** t * h0 + b[None] * series
+    y = (h * Cc[None, None, :]).sum(-1) + Dsk[None, :] * u[None, :]
+    _close(out, y * BIG_Z, what="SSD geometric series: out")
+    _close(hT[0], h[-1], what="SSD geometric series: final state")
+
+
+def pin_ssd_head_indexing(L=None):
+    """Changing the step size or A of ONE head changes the outputs and states of exactly that head's P channels
+    (d = j P + p), and nothing else."""
+    lay, x, z, dt, B, Cm = _ssd_problem(60, H=4, P=3)
+    base = oracle.ssd_prefill(lay, x, z, dt, B, Cm, _lib_override=L)
+    Dn, H, N, W = lay.dims
+    P = lay.headdim
+    for j in range(H):
+        dt2 = dt.copy(); dt2[:, j] += 0.7
+        A2 = lay.A.copy(); A2[j] *= 1.5
+        for alt in (oracle.ssd_prefill(lay, x, z, dt2, B, Cm, _lib_override=L),
+                    oracle.ssd_prefill(oracle.SsdLayer(A2, lay.D, lay.conv_w, lay.conv_b, lay.dt_bias, P, N, flags=lay.flags), x, z, dt, B, Cm, _lib_override=L)):
+            moved = np.abs(alt[0] - base[0]).max(axis=0) > 0
+            want = (np.arange(Dn) // P) == j
+            assert np.array_equal(moved, want), f"head {j}: channels that moved {np.nonzero(moved)[0]}, expected {np.nonzero(want)[0]}"
+            smoved = np.abs(alt[2][0] - base[2][0]).max(axis=1) > 0
+            assert np.array_equal(smoved, want), f"head {j}: states that moved"
+
+
 ALL_PINS = [
     pin_scalar_functions, pin_geometric_series, pin_cumulative_sum, pin_frozen_state, pin_brute_force,
     pin_iir_filter, pin_softplus_and_bias_in_path, pin_conv_impulse, pin_conv_numpy,
     pin_conv_feeds_recurrence, pin_prefill_handoff, pin_prefill_equals_chain, pin_tree_paths, pin_varlen,
     pin_proj_library_matmul, pin_proj_selectors, pin_proj_zero_weights,
+    pin_ssd_is_s6_with_head_constant_A, pin_ssd_geometric_series, pin_ssd_head_indexing,
 ]

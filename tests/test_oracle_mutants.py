@@ -39,6 +39,11 @@ MUTANTS = {
     "proj_sum_drops_last_channel": ("for (int d = 0; d < D; ++d) acc += Wx[(size_t)r * D + d] * u[d];", "for (int d = 0; d + 1 < D; ++d) acc += Wx[(size_t)r * D + d] * u[d];"),
     "proj_ignores_committed_state": ("h[(size_t)d * N + n] = h0 ? h0[(size_t)d * N + n] : 0.0;", "h[(size_t)d * N + n] = 0.0;"),
     "proj_ignores_committed_window": ("win[(size_t)d * (W - 1) + k] = conv0 ? conv0[(size_t)k * D + d] : 0.0;", "win[(size_t)d * (W - 1) + k] = 0.0;"),
+    "ssd_head_of_channel_wrong": ("const int N = L->d_state, W = L->d_conv, j = d / L->headdim;", "const int N = L->d_state, W = L->d_conv, j = d % (L->d_inner / L->headdim);"),
+    "ssd_dt_read_per_channel": ("dt[(size_t)t * H + d / L->headdim], B + (size_t)t * N, C + (size_t)t * N);", "dt[(size_t)t * H + d % H], B + (size_t)t * N, C + (size_t)t * N);"),
+    "ssd_decay_without_delta": ("double decay = exp(delta * L->A[j]);", "double decay = exp(L->A[j]);"),
+    "ssd_bias_per_channel": ("double v = dt + (L->dt_bias ? L->dt_bias[j] : 0.0);", "double v = dt + (L->dt_bias ? L->dt_bias[d % (L->d_inner / L->headdim)] : 0.0);"),
+    "ssd_tree_reads_dt_of_wrong_node": ("dt[a * H + d / L->headdim], B + a * N, C + a * N);", "dt[(size_t)v * H + d / L->headdim], B + a * N, C + a * N);"),
     "delta_softplus_skipped": ("(L->flags & MDO_DT_SOFTPLUS) ? mdo_softplus(v) : v;", "v;"),
 }
 
