@@ -261,12 +261,85 @@ int mdraft_tree_step_proj(const mdraft_layer *layer, const mdraft_cache *cache, 
                           int32_t *dev_status, void *stream);
 
 /*
+ * ---------------------------------------------------------------------------------------------------------
+ * Mamba-2 (SSD) drafter layer.  The paper names Mamba-2 as the model whose advances "directly benefit" the approach
+ * (Section 1, the paragraph before Related Work) and defines nothing about it; what is computed here is the cited
+ * model's recurrence, written like the one at the top of this file with ONE scalar A and ONE step size per head:
+ * the D channels form H = D / P heads of P channels (d = j*P + p),
+ *
+ *     u_t[d]     = SiLU( conv_b[d] + sum_k conv_w[d][k] * x[t-(W-1)+k][d] )
+ *     Delta_t[j] = softplus( dt[t][j] + dt_bias[j] )                         (MDRAFT_DT_SOFTPLUS)
+ *     h_t[d][n]  = exp(Delta_t[j] * A[j]) * h_{t-1}[d][n] + Delta_t[j] * B[t][n] * u_t[d]
+ *     y_t[d]     = sum_n C[t][n] * h_t[d][n] + D[d] * u_t[d]
+ *     out[t][d]  = y_t[d] * SiLU(z[t][d])
+ *
+ * B and C are shared by all heads (one group) and are inputs as given (a block that also convolves them does so
+ * before the call).  Supported: headdim P = 64, d_state N = 128, d_conv 4, bf16 activations, d_inner a multiple of
+ * 64; anything else is MDRAFT_ERR_UNSUPPORTED.  State slots: (D, 128) fp32 + (3, D) bf16 window, in an mdraft_cache
+ * whose strides are sized for N = 128.  flags: MDRAFT_DT_SOFTPLUS only.
+ *
+ * Precision.  The context encode runs the chunk-local sums on the tensor cores (tcgen05, bf16 operands, fp32
+ * accumulation): u * Delta and the masked C.B products are rounded to bf16 on the way into a product, so `out`
+ * carries a relative error of a few 2^-9 before its own rounding to bf16; the incoming state of a chunk and the
+ * operand of the state product are split into a bf16 value plus a bf16 remainder (two products into one
+ * accumulator), so what depends on the state, and the state written to the slot, keep fp32-level accuracy.
+ */
+typedef struct {
+    int32_t d_inner;        /* D */
+    int32_t headdim;        /* P, must be 64 */
+    int32_t d_state;        /* N, must be 128 */
+    int32_t d_conv;         /* W, must be 4 */
+    int32_t act;            /* must be MDRAFT_BF16 */
+    uint32_t flags;         /* MDRAFT_DT_SOFTPLUS or 0 */
+    const float *A;         /* (H) one scalar per head, <= 0 */
+    const float *D;         /* (D) skip weight per channel, or NULL for 0 */
+    const float *conv_w;    /* (D, W) row-major; tap W-1 multiplies the current token */
+    const float *conv_b;    /* (D) or NULL */
+    const float *dt_bias;   /* (H) or NULL */
+} mdraft_ssd_layer;
+
+/*
+ * Context encode of an SSD layer over packed sequences (paper Section 3.1 for the encode; Section 1 for Mamba-2).
+ * Tokens are cut into chunks of 128 that never straddle a sequence; per (head, chunk) the sums inside the chunk are
+ * matrix products on the tensor cores, chunk states are chained by a small scan in between.
+ *   x, z, out : (T, D) bf16, strides ldx, ldz, ldo          dt : (T, H) bf16, stride lddt (elements; any value >= H)
+ *   B, C      : (T, 128) bf16, strides ldb, ldc (multiples of 8 elements, base 16-byte aligned)
+ *   cu_seqlens, init_slot, final_slot, dev_status, stream: as in mdraft_conv_scan_prefill (cu_seqlens may be NULL
+ *   for one sequence)
+ *   workspace : device scratch of at least mdraft_ssd_prefill_workspace_bytes(...) bytes, 256-byte aligned
+ */
+size_t mdraft_ssd_prefill_workspace_bytes(const mdraft_ssd_layer *layer, int32_t total_tokens, int32_t n_seq);
+
+int mdraft_ssd_prefill(const mdraft_ssd_layer *layer, const mdraft_cache *cache, int32_t layer_index,
+                       const void *x, int64_t ldx, const void *z, int64_t ldz, const void *dt, int64_t lddt,
+                       const void *B, int64_t ldb, const void *C, int64_t ldc,
+                       void *out, int64_t ldo,
+                       int32_t total_tokens, int32_t n_seq,
+                       const int32_t *cu_seqlens, const int32_t *init_slot, const int32_t *final_slot,
+                       void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/*
+ * Draft-tree step of an SSD layer: one token for each node of a level, node i from slot parent_slot[i] into slot
+ * node_slot[i] (paper Section 4.1, as mdraft_tree_step).  x, z, out: (M, D); dt: (M, H); B, C: (M, 128).  Levels,
+ * hazards and device-side faults as in mdraft_tree_step; every level is an ordinary launch.  All arithmetic is
+ * fp32 (no tensor cores: one token per node is a memory-bound update of a (D, 128) state).
+ */
+int mdraft_ssd_tree_step(const mdraft_ssd_layer *layer, const mdraft_cache *cache, int32_t layer_index,
+                         const void *x, int64_t ldx, const void *z, int64_t ldz, const void *dt, int64_t lddt,
+                         const void *B, int64_t ldb, const void *C, int64_t ldc,
+                         void *out, int64_t ldo,
+                         int32_t n_nodes, const int32_t *parent_slot, const int32_t *node_slot,
+                         int32_t n_levels, const int32_t *level_offsets,
+                         int32_t *dev_status, void *stream);
+
+/*
  * Accepted-path commit: for j in [0, n_commit) and every layer of the cache,
  * slot dst_slot[j] <- slot src_slot[j] (SSM state and conv window), bit for
  * bit.  After verification the drafter continues from the state of the last
  * accepted node (paper Section 3, speculative decoding loop; Section 4.1).
  * src == dst is a no-op.  A dst that is also some other pair's src is the
- * caller's hazard.  d_inner / act describe the slot contents.
+ * caller's hazard.  d_inner / d_state / act describe the slot contents (d_state 16 for the S6 layers above, 128 for
+ * SSD layers).
  */
 int mdraft_state_commit(const mdraft_cache *cache, int32_t d_inner, int32_t d_state, int32_t d_conv, int32_t act,
                         int32_t n_commit, const int32_t *src_slot, const int32_t *dst_slot,

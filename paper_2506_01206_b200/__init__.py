@@ -11,5 +11,6 @@ from .binding import (  # noqa: F401
     Layer, MdraftError, StateCache, UcbBandit, load_library, mdraft_ucb_reward,
     mdraft_classify_A, mdraft_conv_scan_prefill, mdraft_conv_scan_prefill_noalloc, mdraft_prefill_workspace_bytes,
     NOALLOC_SCRATCH_BYTES,
+    SsdLayer, mdraft_ssd_prefill, mdraft_ssd_prefill_workspace_bytes, mdraft_ssd_tree_step,
     mdraft_state_commit, mdraft_tree_step, mdraft_tree_step_proj, mdraft_version, status_string,
 )

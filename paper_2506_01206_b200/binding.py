@@ -27,6 +27,7 @@ EXPORTS = (
     "mdraft_prefill_workspace_bytes", "mdraft_conv_scan_prefill", "mdraft_conv_scan_prefill_noalloc", "mdraft_tree_step",
     "mdraft_tree_step_proj", "mdraft_state_commit", "mdraft_classify_A", "mdraft_status_string", "mdraft_version",
     "mdraft_ucb_reward", "mdraft_ucb_select", "mdraft_ucb_update",
+    "mdraft_ssd_prefill_workspace_bytes", "mdraft_ssd_prefill", "mdraft_ssd_tree_step",
 )
 
 
@@ -56,6 +57,12 @@ class _PrefillOpts(C.Structure):
 
 class _SelectProj(C.Structure):
     _fields_ = [("W_x", C.c_void_p), ("W_dt", C.c_void_p), ("dt_rank", C.c_int32), ("nodes_per_cluster", C.c_int32)]
+
+
+class _SsdLayer(C.Structure):
+    _fields_ = [("d_inner", C.c_int32), ("headdim", C.c_int32), ("d_state", C.c_int32), ("d_conv", C.c_int32),
+                ("act", C.c_int32), ("flags", C.c_uint32),
+                ("A", C.c_void_p), ("D", C.c_void_p), ("conv_w", C.c_void_p), ("conv_b", C.c_void_p), ("dt_bias", C.c_void_p)]
 
 
 class _Ucb(C.Structure):
@@ -108,6 +115,16 @@ def load_library(path: Optional[str] = None):
     lib.mdraft_ucb_select.argtypes = [C.POINTER(_Ucb), C.POINTER(i32)]
     lib.mdraft_ucb_update.restype = C.c_int
     lib.mdraft_ucb_update.argtypes = [C.POINTER(_Ucb), i32, i32, i32]
+    lib.mdraft_ssd_prefill_workspace_bytes.restype = C.c_size_t
+    lib.mdraft_ssd_prefill_workspace_bytes.argtypes = [C.POINTER(_SsdLayer), i32, i32]
+    lib.mdraft_ssd_prefill.restype = C.c_int
+    lib.mdraft_ssd_prefill.argtypes = [C.POINTER(_SsdLayer), C.POINTER(_Cache), i32,
+                                       vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
+                                       i32, i32, vp, vp, vp, vp, C.c_size_t, vp, vp]
+    lib.mdraft_ssd_tree_step.restype = C.c_int
+    lib.mdraft_ssd_tree_step.argtypes = [C.POINTER(_SsdLayer), C.POINTER(_Cache), i32,
+                                         vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64,
+                                         i32, vp, vp, i32, C.POINTER(i32), vp, vp]
     if path is None:
         _lib = lib
     return lib
@@ -394,3 +411,87 @@ class UcbBandit:
 
 def mdraft_ucb_reward(lambda_gamma: float, draft_len: int, n_accept: int) -> float:
     return float(load_library().mdraft_ucb_reward(float(lambda_gamma), int(draft_len), int(n_accept)))
+
+
+# ---------------------------------------------------------------- Mamba-2 (SSD) layer
+@dataclass
+class SsdLayer:
+    """Constants of an SSD layer on the device (fp32): A (H,), dt_bias (H,), D (D,), conv taps (D, W)."""
+    A: torch.Tensor
+    D: Optional[torch.Tensor]
+    conv_w: torch.Tensor
+    conv_b: Optional[torch.Tensor]
+    dt_bias: Optional[torch.Tensor]
+    headdim: int = 64
+    d_state: int = 128
+    flags: int = MDRAFT_DT_SOFTPLUS
+
+    def __post_init__(self):
+        Dn, W = self.conv_w.shape
+        H = int(self.A.numel())
+        if H * self.headdim != Dn:
+            raise ValueError("A must hold one value per head of `headdim` channels")
+        _f32(self.A, H, "A"); _f32(self.conv_w, Dn * W, "conv_w")
+        _f32(self.D, Dn, "D"); _f32(self.conv_b, Dn, "conv_b"); _f32(self.dt_bias, H, "dt_bias")
+        self.d_inner, self.n_heads, self.d_conv = int(Dn), H, int(W)
+
+    def c(self, flags: Optional[int] = None) -> _SsdLayer:
+        return _SsdLayer(self.d_inner, self.headdim, self.d_state, self.d_conv, MDRAFT_BF16,
+                         self.flags if flags is None else int(flags),
+                         self.A.data_ptr(), 0 if self.D is None else self.D.data_ptr(), self.conv_w.data_ptr(),
+                         0 if self.conv_b is None else self.conv_b.data_ptr(),
+                         0 if self.dt_bias is None else self.dt_bias.data_ptr())
+
+
+def mdraft_ssd_prefill_workspace_bytes(layer: SsdLayer, total_tokens: int, n_seq: int) -> int:
+    cl = layer.c()
+    return int(load_library().mdraft_ssd_prefill_workspace_bytes(C.byref(cl), int(total_tokens), int(n_seq)))
+
+
+def mdraft_ssd_prefill(layer: SsdLayer, cache: Optional[StateCache], layer_index: int, x, z, dt, B, Cm, out,
+                       cu_seqlens: Optional[torch.Tensor], init_slot: Optional[torch.Tensor] = None,
+                       final_slot: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                       dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None) -> None:
+    lib = load_library()
+    cl = layer.c(flags)
+    cc = cache.c() if cache is not None else None
+    px, ldx = _mat(x, "x"); pz, ldz = _mat(z, "z"); pdt, lddt = _mat(dt, "dt")
+    pB, ldb = _mat(B, "B"); pC, ldc = _mat(Cm, "C"); po, ldo = _mat(out, "out")
+    T = int(x.shape[0])
+    n_seq = 1 if cu_seqlens is None else int(cu_seqlens.numel()) - 1
+    if cu_seqlens is not None and cu_seqlens.dtype != torch.int32:
+        raise TypeError("cu_seqlens must be int32")
+    for t, nm in ((init_slot, "init_slot"), (final_slot, "final_slot")):
+        if t is not None and (t.dtype != torch.int32 or t.numel() != n_seq):
+            raise TypeError(f"{nm} must be int32 with one entry per sequence")
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (C.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    rc = lib.mdraft_ssd_prefill(C.byref(cl), C.byref(cc) if cc is not None else None, int(layer_index),
+                                px, ldx, pz, ldz, pdt, lddt, pB, ldb, pC, ldc, po, ldo, T, n_seq,
+                                _ptr(cu_seqlens), _ptr(init_slot), _ptr(final_slot), ws_ptr, ws_bytes, _ptr(dev_status), _stream_ptr(stream))
+    if rc != 0:
+        raise MdraftError(rc, "mdraft_ssd_prefill")
+
+
+def mdraft_ssd_tree_step(layer: SsdLayer, cache: StateCache, layer_index: int, x, z, dt, B, Cm, out,
+                         parent_slot: torch.Tensor, node_slot: torch.Tensor, level_offsets: Optional[Sequence[int]] = None,
+                         dev_status: Optional[torch.Tensor] = None, stream=None, flags: Optional[int] = None) -> None:
+    lib = load_library()
+    cl = layer.c(flags)
+    cc = cache.c()
+    px, ldx = _mat(x, "x"); pz, ldz = _mat(z, "z"); pdt, lddt = _mat(dt, "dt")
+    pB, ldb = _mat(B, "B"); pC, ldc = _mat(Cm, "C"); po, ldo = _mat(out, "out")
+    M = int(x.shape[0])
+    if parent_slot.dtype != torch.int32 or node_slot.dtype != torch.int32:
+        raise TypeError("slot index arrays must be int32")
+    if parent_slot.numel() != M or node_slot.numel() != M:
+        raise ValueError("one parent slot and one node slot per node")
+    if level_offsets is None:
+        n_levels, lo = 1, None
+    else:
+        n_levels = len(level_offsets) - 1
+        lo = (C.c_int32 * (n_levels + 1))(*[int(v) for v in level_offsets])
+    rc = lib.mdraft_ssd_tree_step(C.byref(cl), C.byref(cc), int(layer_index),
+                                  px, ldx, pz, ldz, pdt, lddt, pB, ldb, pC, ldc, po, ldo,
+                                  M, _ptr(parent_slot), _ptr(node_slot), n_levels, lo, _ptr(dev_status), _stream_ptr(stream))
+    if rc != 0:
+        raise MdraftError(rc, "mdraft_ssd_tree_step")

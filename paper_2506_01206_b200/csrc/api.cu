@@ -8,6 +8,7 @@
 #include "commit.cuh"
 #include "common.cuh"
 #include "prefill.cuh"
+#include "ssd.cuh"
 #include "tree_proj.cuh"
 #include "tree_step.cuh"
 
@@ -31,10 +32,10 @@ int check_layer(const mdraft_layer* L) {
     return MDRAFT_OK;
 }
 
-int check_cache(const mdraft_cache* c, int d_inner, int act, int layer_index) {
+int check_cache(const mdraft_cache* c, int d_inner, int act, int layer_index, int d_state = kN) {
     if (!c || !c->ssm || !c->conv) return MDRAFT_ERR_INVALID_ARG;
     if (c->n_layers <= 0 || c->n_slots <= 0 || layer_index < 0 || layer_index >= c->n_layers) return MDRAFT_ERR_INVALID_ARG;
-    const int64_t ssm_elems = (int64_t)d_inner * kN, conv_elems = (int64_t)(kW - 1) * d_inner;
+    const int64_t ssm_elems = (int64_t)d_inner * d_state, conv_elems = (int64_t)(kW - 1) * d_inner;
     if (c->ssm_slot_stride < ssm_elems || c->conv_slot_stride < conv_elems) return MDRAFT_ERR_INVALID_ARG;
     if (c->n_layers > 1 && (c->ssm_layer_stride < 0 || c->conv_layer_stride < 0)) return MDRAFT_ERR_INVALID_ARG;
     const size_t es = elem_size(act);
@@ -348,8 +349,8 @@ int mdraft_state_commit(const mdraft_cache* cache, int32_t d_inner, int32_t d_st
                         int32_t n_commit, const int32_t* src_slot, const int32_t* dst_slot, int32_t* dev_status,
                         void* stream) {
     if (d_inner <= 0 || n_commit < 0) return MDRAFT_ERR_INVALID_ARG;
-    if (d_state != kN || d_conv != kW || (d_inner % 8) != 0 || (act != MDRAFT_F32 && act != MDRAFT_BF16)) return MDRAFT_ERR_UNSUPPORTED;
-    int rc = check_cache(cache, d_inner, act, 0);
+    if ((d_state != kN && d_state != kSsdN) || d_conv != kW || (d_inner % 8) != 0 || (act != MDRAFT_F32 && act != MDRAFT_BF16)) return MDRAFT_ERR_UNSUPPORTED;
+    int rc = check_cache(cache, d_inner, act, 0, d_state);
     if (rc) return rc;
     if (n_commit == 0) return MDRAFT_OK;
     if (!src_slot || !dst_slot) return MDRAFT_ERR_INVALID_ARG;
@@ -359,7 +360,7 @@ int mdraft_state_commit(const mdraft_cache* cache, int32_t d_inner, int32_t d_st
     a.conv = static_cast<char*>(cache->conv);
     a.ssm_layer_bytes = cache->ssm_layer_stride * 4; a.ssm_slot_bytes_stride = cache->ssm_slot_stride * 4;
     a.conv_layer_bytes = cache->conv_layer_stride * es; a.conv_slot_bytes_stride = cache->conv_slot_stride * es;
-    a.ssm_bytes = (int64_t)d_inner * kN * 4; a.conv_bytes = (int64_t)(kW - 1) * d_inner * es;
+    a.ssm_bytes = (int64_t)d_inner * d_state * 4; a.conv_bytes = (int64_t)(kW - 1) * d_inner * es;
     a.n_layers = cache->n_layers; a.n_slots = cache->n_slots; a.dev_status = dev_status;
     if (a.n_layers > 65535) return MDRAFT_ERR_UNSUPPORTED;
     for (int off = 0; off < n_commit; off += 65535) {
@@ -382,6 +383,156 @@ int mdraft_classify_A(const float* A, int32_t d_inner, int32_t d_state, int32_t*
     if (cudaStreamSynchronize(st) != cudaSuccess) return MDRAFT_ERR_CUDA;
     *is_powers = host[0] == 0;
     if (is_nonpositive) *is_nonpositive = host[1] == 0;
+    return MDRAFT_OK;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------- SSD layer
+namespace {
+
+int check_ssd_layer(const mdraft_ssd_layer* L) {
+    if (!L || !L->A || !L->conv_w) return MDRAFT_ERR_INVALID_ARG;
+    if (L->d_inner <= 0) return MDRAFT_ERR_INVALID_ARG;
+    if (L->headdim != kSsdP || L->d_state != kSsdN || L->d_conv != kW || (L->d_inner % kSsdP) != 0 || L->act != MDRAFT_BF16)
+        return MDRAFT_ERR_UNSUPPORTED;
+    if (L->flags & ~(uint32_t)MDRAFT_DT_SOFTPLUS) return MDRAFT_ERR_INVALID_ARG;
+    if (!aligned16(L->conv_w)) return MDRAFT_ERR_MISALIGNED;
+    return MDRAFT_OK;
+}
+
+SsdLayerDev ssd_layer_dev(const mdraft_ssd_layer* L) {
+    SsdLayerDev d;
+    d.A = L->A; d.D = L->D; d.conv_w = L->conv_w; d.conv_b = L->conv_b; d.dt_bias = L->dt_bias;
+    d.d_inner = L->d_inner; d.n_heads = L->d_inner / L->headdim; d.flags = L->flags;
+    return d;
+}
+
+struct SsdPlan {
+    int n_chunks_bound;
+    size_t off_S, off_decay, off_hin, bytes;
+};
+
+SsdPlan plan_ssd(const mdraft_ssd_layer* L, int T, int n_seq) {
+    SsdPlan pl;
+    const size_t H = (size_t)(L->d_inner / L->headdim);
+    pl.n_chunks_bound = n_seq + T / kSsdQ;
+    const size_t per_chunk = H * kSsdP * kSsdN;
+    pl.off_S = 0;
+    pl.off_decay = align_up(pl.off_S + (size_t)pl.n_chunks_bound * per_chunk * sizeof(float), 256);
+    pl.off_hin = align_up(pl.off_decay + (size_t)pl.n_chunks_bound * H * sizeof(float), 256);
+    pl.bytes = align_up(pl.off_hin + (size_t)pl.n_chunks_bound * per_chunk * 2 * 2, 256);   // bf16 value + bf16 remainder
+    return pl;
+}
+
+// Descriptor of a (rows x cols) row-major bf16 matrix read in boxes of box_cols x 128 rows.
+bool encode_ssd_matrix(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols) {
+    PFN_cuTensorMapEncodeTiled enc = tensor_map_encoder();
+    if (!enc) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)kSsdQ};
+    cuuint32_t estride[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mdraft_ssd_prefill_workspace_bytes(const mdraft_ssd_layer* layer, int32_t total_tokens, int32_t n_seq) {
+    if (check_ssd_layer(layer) != MDRAFT_OK || total_tokens <= 0 || n_seq <= 0) return 0;
+    return plan_ssd(layer, total_tokens, n_seq).bytes;
+}
+
+int mdraft_ssd_prefill(const mdraft_ssd_layer* layer, const mdraft_cache* cache, int32_t layer_index, const void* x, int64_t ldx,
+                       const void* z, int64_t ldz, const void* dt, int64_t lddt, const void* B, int64_t ldb, const void* C,
+                       int64_t ldc, void* out, int64_t ldo, int32_t total_tokens, int32_t n_seq, const int32_t* cu_seqlens,
+                       const int32_t* init_slot, const int32_t* final_slot, void* workspace, size_t workspace_bytes,
+                       int32_t* dev_status, void* stream) {
+    int rc = check_ssd_layer(layer);
+    if (rc) return rc;
+    if (total_tokens < 0 || n_seq < 0) return MDRAFT_ERR_INVALID_ARG;
+    if (init_slot || final_slot || cache) {
+        rc = check_cache(cache, layer->d_inner, layer->act, layer_index, kSsdN);
+        if (rc) return rc;
+    }
+    if (n_seq == 0) return MDRAFT_OK;
+    if (!cu_seqlens && n_seq != 1) return MDRAFT_ERR_INVALID_ARG;
+    const int D = layer->d_inner, H = D / layer->headdim;
+    const bool have_rows = total_tokens > 0;
+    if ((rc = check_matrix(x, ldx, D, MDRAFT_BF16, have_rows))) return rc;
+    if ((rc = check_matrix(z, ldz, D, MDRAFT_BF16, have_rows))) return rc;
+    if ((rc = check_matrix(out, ldo, D, MDRAFT_BF16, have_rows))) return rc;
+    if ((rc = check_matrix(B, ldb, kSsdN, MDRAFT_BF16, have_rows))) return rc;
+    if ((rc = check_matrix(C, ldc, kSsdN, MDRAFT_BF16, have_rows))) return rc;
+    if (have_rows && (!dt || lddt < H)) return MDRAFT_ERR_INVALID_ARG;
+    const SsdPlan pl = plan_ssd(layer, have_rows ? total_tokens : 1, n_seq);
+    if (!workspace || workspace_bytes < pl.bytes) return MDRAFT_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MDRAFT_ERR_MISALIGNED;
+    if (pl.n_chunks_bound > 65535) return MDRAFT_ERR_UNSUPPORTED;
+
+    SsdPrefillArgs a;
+    a.L = ssd_layer_dev(layer);
+    if (cache) a.pool = pool_dev(cache, MDRAFT_BF16, layer_index);
+    else { a.pool.ssm = nullptr; a.pool.conv = nullptr; a.pool.ssm_slot_stride = 0; a.pool.conv_slot_stride = 0; a.pool.n_slots = 0; }
+    a.x = static_cast<const __nv_bfloat16*>(x); a.z = static_cast<const __nv_bfloat16*>(z); a.dt = static_cast<const __nv_bfloat16*>(dt);
+    a.B = static_cast<const __nv_bfloat16*>(B); a.C = static_cast<const __nv_bfloat16*>(C); a.out = static_cast<__nv_bfloat16*>(out);
+    a.ldx = ldx; a.ldz = ldz; a.lddt = lddt; a.ldb = ldb; a.ldc = ldc; a.ldo = ldo;
+    a.T = total_tokens; a.n_seq = n_seq; a.n_chunks_bound = pl.n_chunks_bound;
+    a.cu = cu_seqlens; a.init_slot = init_slot; a.final_slot = final_slot;
+    char* ws = static_cast<char*>(workspace);
+    a.ws_S = reinterpret_cast<float*>(ws + pl.off_S);
+    a.ws_decay = reinterpret_cast<float*>(ws + pl.off_decay);
+    a.ws_hin = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_hin);
+    a.dev_status = dev_status;
+    SsdMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (have_rows) {
+        if (!encode_ssd_matrix(&maps.x, x, total_tokens, D, ldx, kSsdP) || !encode_ssd_matrix(&maps.z, z, total_tokens, D, ldz, kSsdP) ||
+            !encode_ssd_matrix(&maps.B, B, total_tokens, kSsdN, ldb, 8) || !encode_ssd_matrix(&maps.C, C, total_tokens, kSsdN, ldc, 8))
+            return MDRAFT_ERR_CUDA;
+    }
+    return launch_ssd_prefill(a, maps, static_cast<cudaStream_t>(stream)) == cudaSuccess ? MDRAFT_OK : MDRAFT_ERR_CUDA;
+}
+
+int mdraft_ssd_tree_step(const mdraft_ssd_layer* layer, const mdraft_cache* cache, int32_t layer_index, const void* x, int64_t ldx,
+                         const void* z, int64_t ldz, const void* dt, int64_t lddt, const void* B, int64_t ldb, const void* C,
+                         int64_t ldc, void* out, int64_t ldo, int32_t n_nodes, const int32_t* parent_slot, const int32_t* node_slot,
+                         int32_t n_levels, const int32_t* level_offsets, int32_t* dev_status, void* stream) {
+    int rc = check_ssd_layer(layer);
+    if (rc) return rc;
+    if ((rc = check_cache(cache, layer->d_inner, layer->act, layer_index, kSsdN))) return rc;
+    if (n_nodes < 0 || n_levels < 0) return MDRAFT_ERR_INVALID_ARG;
+    if (n_nodes == 0) return MDRAFT_OK;
+    if (!parent_slot || !node_slot) return MDRAFT_ERR_INVALID_ARG;
+    if (!level_offsets && n_levels > 1) return MDRAFT_ERR_INVALID_ARG;
+    if (level_offsets) {
+        if (n_levels < 1 || level_offsets[0] != 0 || level_offsets[n_levels] != n_nodes) return MDRAFT_ERR_INVALID_ARG;
+        for (int l = 0; l < n_levels; ++l)
+            if (level_offsets[l + 1] < level_offsets[l]) return MDRAFT_ERR_INVALID_ARG;
+    }
+    const int D = layer->d_inner, H = D / layer->headdim;
+    if ((rc = check_matrix(x, ldx, D, MDRAFT_BF16, true))) return rc;
+    if ((rc = check_matrix(z, ldz, D, MDRAFT_BF16, true))) return rc;
+    if ((rc = check_matrix(out, ldo, D, MDRAFT_BF16, true))) return rc;
+    if ((rc = check_matrix(B, ldb, kSsdN, MDRAFT_BF16, true))) return rc;
+    if ((rc = check_matrix(C, ldc, kSsdN, MDRAFT_BF16, true))) return rc;
+    if (!dt || lddt < H) return MDRAFT_ERR_INVALID_ARG;
+    SsdStepArgs a;
+    a.L = ssd_layer_dev(layer);
+    a.pool = pool_dev(cache, MDRAFT_BF16, layer_index);
+    a.x = static_cast<const __nv_bfloat16*>(x); a.z = static_cast<const __nv_bfloat16*>(z); a.dt = static_cast<const __nv_bfloat16*>(dt);
+    a.B = static_cast<const __nv_bfloat16*>(B); a.C = static_cast<const __nv_bfloat16*>(C); a.out = static_cast<__nv_bfloat16*>(out);
+    a.ldx = ldx; a.ldz = ldz; a.lddt = lddt; a.ldb = ldb; a.ldc = ldc; a.ldo = ldo;
+    a.parent_slot = parent_slot; a.node_slot = node_slot; a.dev_status = dev_status;
+    const int levels = level_offsets ? n_levels : 1;
+    for (int l = 0; l < levels; ++l) {
+        a.lvl_begin = level_offsets ? level_offsets[l] : 0;
+        a.lvl_end = level_offsets ? level_offsets[l + 1] : n_nodes;
+        if (launch_ssd_step(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MDRAFT_ERR_CUDA;
+    }
     return MDRAFT_OK;
 }
 

@@ -1,0 +1,521 @@
+// Context encode of a Mamba-2 (SSD) layer: conv1d+SiLU -> Delta -> recurrence with one scalar A per head -> gate.
+//
+// With a scalar decay per head the recurrence of a chunk of Q tokens turns into matrix products (the "state-space
+// duality" form).  With cs_t = sum_{r <= t} Delta_r A (the running log-decay inside the chunk), for a head of P channels:
+//
+//     y_t = sum_{s <= t} (C_t . B_s) exp(cs_t - cs_s) Delta_s u_s      (inside the chunk:  (G o L) Xd,  G = C B^T)
+//           + exp(cs_t) C_t . h_in                                      (from the incoming state:  C H_in^T, row-scaled)
+//     S   = sum_s exp(cs_end - cs_s) Delta_s u_s (x) B_s                (what the chunk adds to a zero state)
+//     h_out = exp(cs_end) h_in + S
+//
+// Three stream-ordered kernels, none waiting on another block:
+//   1. ssd_chunk_state: per (head, chunk) S^T = B^T Xw on the tensor cores (tcgen05.mma, bf16 operands, fp32 accumulator
+//      in tensor memory); Xw is split into a bf16 value and a bf16 remainder (two products into one accumulator) so that
+//      the state keeps fp32-level accuracy.
+//   2. ssd_state_passing: per (channel, 8 states) the chunk states of a sequence are chained in token order; every
+//      chunk's incoming state is left in the operand layout the next kernel wants, the final state goes to its slot.
+//   3. ssd_chunk_scan: per (head, chunk) G = C B^T, the causal decay mask applied to G on its way from tensor memory to
+//      shared memory, Y = (G o L) Xd and C H_in^T on the tensor cores, then skip term, gate and store.
+//
+// Operands live in shared memory in the tensor core's canonical un-swizzled layout: 16-byte units of 8 bf16 values,
+// 8 units = one 8 x 8 "core matrix" of 128 contiguous bytes; one descriptor field gives the byte step between core
+// matrices along the contraction index, the other along the row index.  A TMA box of 8 columns x 128 rows of a
+// row-major matrix lands exactly as one column of core matrices, so B and C arrive in operand form without a pass
+// over them, both as "K-major" (G: contraction over the state index) and as "MN-major" (S: contraction over tokens).
+// All waits on mbarriers are bounded (MDRAFT_DEV_WAIT_EXPIRED); tensor memory is freed on every path.
+#include "chunk_map.cuh"
+#include "common.cuh"
+#include "ssd.cuh"
+
+namespace mdraft {
+
+namespace {
+
+constexpr int P = kSsdP, N = kSsdN, Q = kSsdQ;
+constexpr int kThreads = 128;                 // one thread per chunk row / accumulator lane
+constexpr uint32_t kColBytes = Q * 16;        // one 8-wide column of core matrices over 128 rows: 2048 bytes
+constexpr uint32_t kXdColBytes = Q * 16 + 16; // the same for the thread-written Xd / Xw operand, padded against bank conflicts
+constexpr uint32_t kHinColBytes = P * 16;     // H_in: 64 rows
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes + kOverstateTx) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kPollNs) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_box(void* dst, const CUtensorMap* map, int col, int row, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_u32(dst)),
+                 "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(row), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+                 "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// Tensor memory: allocation (one warp), release, and the accumulator loads (a warp reads the 32 lanes it owns).
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot_in_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot_in_smem)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_free(uint32_t base, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory operand descriptor, un-swizzled canonical layout.  `lead` / `stride` are the two byte steps between core
+// matrices: for a K-major operand lead = along the contraction index, stride = along rows; for an MN-major operand
+// lead = along the contraction index (groups of 8), stride = along the row index (groups of 8).
+__device__ __forceinline__ uint64_t operand_desc(uint32_t saddr, uint32_t lead, uint32_t stride) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lead >> 4) & 0x3FFFu) << 16) | ((uint64_t)((stride >> 4) & 0x3FFFu) << 32) |
+           (1ull << 46);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n; bit 15 / 16 = A / B operand is MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+// D (tensor memory) (+)= A (smem) * B (smem), one instruction of contraction length 16; issued by ONE thread.
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate ? 1u : 0u), "r"(0u)
+        : "memory");
+}
+// All tensor-core work issued so far by this thread arrives on the mbarrier when it has completed.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// ---------------------------------------------------------------- what both tensor-core kernels share
+// Per-row scalars of a chunk: step size and running log-decay.  Thread t = row t; rows past the chunk's end get a
+// step size of 0 (no decay, no input).  Leaves delta[t], cs[t] (natural log) and csl[t] = cs[t] * log2(e) in shared memory.
+struct RowScalars {
+    float delta[Q];
+    float cs[Q];
+    float csl[Q];
+    float warp_sum[4];
+};
+
+__device__ __forceinline__ void row_scalars(RowScalars& rs, const SsdPrefillArgs& p, int head, int t0, int rows) {
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    float delta = 0.0f;
+    if (t < rows) {
+        const float v = __bfloat162float(p.dt[(size_t)(t0 + t) * p.lddt + head]) + (p.L.dt_bias ? __ldg(p.L.dt_bias + head) : 0.0f);
+        delta = (p.L.flags & MDRAFT_DT_SOFTPLUS) ? softplus(v) : v;
+    }
+    float la = delta * __ldg(p.L.A + head);
+    // inclusive scan over the 128 rows: inside the warp by shuffles, across the four warps through shared memory
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float up = __shfl_up_sync(0xffffffffu, la, o);
+        if (lane >= o) la += up;
+    }
+    if (lane == 31) rs.warp_sum[warp] = la;
+    __syncthreads();
+    float before = 0.0f;
+    for (int w = 0; w < warp; ++w) before += rs.warp_sum[w];
+    la += before;
+    rs.delta[t] = delta;
+    rs.cs[t] = la;
+    rs.csl[t] = la * kLog2e;
+    __syncthreads();
+}
+
+// The three rows before the chunk, as rows 0..2 of the extended x tile (rows 3.. are the TMA box): the sequence's own
+// tokens, or the window of its starting slot, or zeros.  Threads 0..95, one bf16 pair each.
+__device__ __forceinline__ void load_halo(__nv_bfloat16* xs_ext, const SsdPrefillArgs& p, const ChunkInfo& ci, int head, int islot) {
+    const int t = threadIdx.x;
+    if (t >= 3 * 32) return;
+    const int j = t >> 5, lane = t & 31;
+    const int d = head * P + 2 * lane;
+    uint32_t v = 0u;
+    if (ci.k > 0) v = *reinterpret_cast<const uint32_t*>(p.x + (size_t)(ci.t0 - 3 + j) * p.ldx + d);
+    else if (islot >= 0) v = *reinterpret_cast<const uint32_t*>(static_cast<const __nv_bfloat16*>(p.pool.conv) + (size_t)islot * p.pool.conv_slot_stride + (size_t)j * p.L.d_inner + d);
+    *reinterpret_cast<uint32_t*>(xs_ext + j * P + 2 * lane) = v;
+}
+
+// conv + SiLU of the warp's 32 rows for this lane's channel pair; calls f(row, u_lo, u_hi) for every row.
+template <typename F>
+__device__ __forceinline__ void conv_rows(const __nv_bfloat16* xs_ext, const SsdLayerDev& L, int head, F&& f) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int d = head * P + 2 * lane;
+    const float4 wa = __ldg(reinterpret_cast<const float4*>(L.conv_w + (size_t)d * kW));
+    const float4 wb = __ldg(reinterpret_cast<const float4*>(L.conv_w + (size_t)(d + 1) * kW));
+    const float ba = L.conv_b ? __ldg(L.conv_b + d) : 0.0f, bb = L.conv_b ? __ldg(L.conv_b + d + 1) : 0.0f;
+    const uint32_t* col = reinterpret_cast<const uint32_t*>(xs_ext) + lane;   // row r of the chunk is extended row r + 3
+    const int r0 = warp * 32;
+    uint32_t w0 = col[(r0 + 0) * (P / 2)], w1 = col[(r0 + 1) * (P / 2)], w2 = col[(r0 + 2) * (P / 2)];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const uint32_t xv = col[(r0 + i + 3) * (P / 2)];
+        float a = fmaf(wa.x, bf_lo(w0), ba), b = fmaf(wb.x, bf_hi(w0), bb);
+        a = fmaf(wa.y, bf_lo(w1), a); b = fmaf(wb.y, bf_hi(w1), b);
+        a = fmaf(wa.z, bf_lo(w2), a); b = fmaf(wb.z, bf_hi(w2), b);
+        a = fmaf(wa.w, bf_lo(xv), a); b = fmaf(wb.w, bf_hi(xv), b);
+        w0 = w1; w1 = w2; w2 = xv;
+        f(r0 + i, silu(a), silu(b));
+    }
+}
+
+// ---------------------------------------------------------------- kernel 1: what a chunk adds to a zero state
+struct StateSmem {
+    __nv_bfloat16 Bt[N / 8][Q][8];                        // B rows of the chunk, one TMA box per 8 states
+    unsigned char xw_hi[(P / 8) * kXdColBytes];           // Xw = Delta exp(cs_end - cs) u, bf16 value ...
+    unsigned char xw_lo[(P / 8) * kXdColBytes];           // ... and bf16 remainder
+    __nv_bfloat16 xs_ext[(Q + 3) * P];                    // 3 rows before the chunk + the x box
+    RowScalars rs;
+    uint64_t bar_tma, bar_mma;
+    uint32_t tmem_base;
+};
+
+__global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
+    extern __shared__ __align__(1024) unsigned char s_raw[];
+    StateSmem& sm = *reinterpret_cast<StateSmem*>(s_raw + ((1024u - (smem_u32(s_raw) & 1023u)) & 1023u));
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads;
+    const ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, Q, cidx);
+    if (ci.seq < 0) return;
+    const int islot = load_slot(p.init_slot, ci.seq), fslot = load_slot(p.final_slot, ci.seq);
+    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;   // reported by the state-passing kernel
+    const int rows = ci.t1 - ci.t0;
+
+    if (tid == 0) {
+        mbar_init(&sm.bar_tma, 1);
+        mbar_init(&sm.bar_mma, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(&sm.bar_tma, Q * P * 2 + Q * N * 2);
+        tma_box(sm.xs_ext + 3 * P, &maps.x, head * P, ci.t0, &sm.bar_tma);
+#pragma unroll
+        for (int c = 0; c < N / 8; ++c) tma_box(&sm.Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_tma);
+    }
+    if (warp == 0) { tmem_alloc(&sm.tmem_base, 64); tc_fence_before(); }
+    load_halo(sm.xs_ext, p, ci, head, islot);
+    row_scalars(sm.rs, p, head, ci.t0, rows);   // two block-wide barriers inside: barrier init and tmem_base are visible after it
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    bool ok = mbar_wait_bounded(&sm.bar_tma, 0u);
+    if (ok) {
+        const float cs_end_l = sm.rs.csl[Q - 1];
+        conv_rows(sm.xs_ext, p.L, head, [&](int r, float ua, float ub) {
+            const float wgt = r < rows ? sm.rs.delta[r] * ex2(cs_end_l - sm.rs.csl[r]) : 0.0f;
+            const float va = r < rows ? wgt * ua : 0.0f, vb = r < rows ? wgt * ub : 0.0f;
+            const uint32_t hi = pack_bf(va, vb);
+            const uint32_t lo = pack_bf(va - bf_lo(hi), vb - bf_hi(hi));
+            const uint32_t off = (uint32_t)(lane >> 2) * kXdColBytes + (uint32_t)r * 16u + (uint32_t)(lane & 3) * 4u;
+            *reinterpret_cast<uint32_t*>(sm.xw_hi + off) = hi;
+            *reinterpret_cast<uint32_t*>(sm.xw_lo + off) = lo;
+        });
+    }
+    fence_async_smem();   // the operand written by threads must be visible to the tensor core's reads
+    const bool all_ok = !__syncthreads_or(!ok);
+    if (all_ok && tid == 0) {
+        tc_fence_after();
+        // S^T (n x p) = sum over tokens: A operand = B^T read MN-major out of the TMA boxes, B operand = Xw MN-major.
+        constexpr uint32_t idesc = instr_desc(P, true, true);
+        const uint32_t a0 = smem_u32(&sm.Bt[0][0][0]), bh = smem_u32(sm.xw_hi), bl = smem_u32(sm.xw_lo);
+#pragma unroll
+        for (int k = 0; k < Q / 16; ++k)
+            mma_bf16(tmem, operand_desc(a0 + k * 256, 128, kColBytes), operand_desc(bh + k * 256, 128, kXdColBytes), idesc, k > 0);
+#pragma unroll
+        for (int k = 0; k < Q / 16; ++k)
+            mma_bf16(tmem, operand_desc(a0 + k * 256, 128, kColBytes), operand_desc(bl + k * 256, 128, kXdColBytes), idesc, true);
+        mma_commit(&sm.bar_mma);
+    }
+    bool done = all_ok && mbar_wait_bounded(&sm.bar_mma, 0u);
+    if (done) {
+        tc_fence_after();
+        // thread n holds row n of S^T: 64 values, one per channel of the head; stores are contiguous across threads
+        float* dst = p.ws_S + ((size_t)cidx * H + head) * P * N + tid;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            float v[32];
+            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + half * 32, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) dst[(size_t)(half * 32 + j) * N] = v[j];
+        }
+        if (tid == 0) p.ws_decay[(size_t)cidx * H + head] = sm.rs.cs[Q - 1];
+    } else if (tid == 0) {
+        flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
+        if (!ok) mbar_wait_bounded(&sm.bar_tma, 0u);   // the copies target this block's shared memory: one more bounded chance
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_free(tmem, 64);
+}
+
+// ---------------------------------------------------------------- kernel 2: chain the chunk states of a sequence
+// Thread = (channel d, group of 8 states).  Walks the sequence's chunks in order: writes the chunk's incoming state as
+// bf16 (a value and a remainder) in the operand layout [state group][channel of the head][8], then h <- exp(chunk decay) h + S.
+__global__ void __launch_bounds__(256) ssd_state_passing_kernel(const SsdPrefillArgs p) {
+    const int D = p.L.d_inner, H = p.L.n_heads;
+    const int s = blockIdx.y;
+    const int idx = blockIdx.x * 256 + threadIdx.x;
+    int first, nck;
+    seq_chunks(p.cu, p.n_seq, p.T, Q, s, first, nck);   // whole warps call this
+    // malformed offsets: the sequence has no chunk and is skipped
+    if (p.cu && blockIdx.x == 0 && threadIdx.x == 0) {
+        const int lo = __ldg(p.cu + s), hi = __ldg(p.cu + s + 1);
+        if (lo < 0 || hi < lo || hi > p.T) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);
+    }
+    const int islot = load_slot(p.init_slot, s), fslot = load_slot(p.final_slot, s);
+    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+        return;
+    }
+    if (idx >= D * (N / 8)) return;
+    const int g = idx % (N / 8), d = idx / (N / 8), head = d / P, ch = d % P;   // consecutive threads: consecutive state groups of one channel
+    float h[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) h[i] = 0.0f;
+    if (islot >= 0) {
+        const float4* src = reinterpret_cast<const float4*>(p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)d * N + g * 8);
+        const float4 a = src[0], b = src[1];
+        h[0] = a.x; h[1] = a.y; h[2] = a.z; h[3] = a.w; h[4] = b.x; h[5] = b.y; h[6] = b.z; h[7] = b.w;
+    }
+    for (int c = first; c < first + nck; ++c) {
+        const size_t ch_head = (size_t)c * H + head;
+        // bf16 value and bf16 remainder of the incoming state: two operands, so that the product with C sees ~16 mantissa bits
+        uint4 hi4, lo4;
+        hi4.x = pack_bf(h[0], h[1]); hi4.y = pack_bf(h[2], h[3]); hi4.z = pack_bf(h[4], h[5]); hi4.w = pack_bf(h[6], h[7]);
+        lo4.x = pack_bf(h[0] - bf_lo(hi4.x), h[1] - bf_hi(hi4.x)); lo4.y = pack_bf(h[2] - bf_lo(hi4.y), h[3] - bf_hi(hi4.y));
+        lo4.z = pack_bf(h[4] - bf_lo(hi4.z), h[5] - bf_hi(hi4.z)); lo4.w = pack_bf(h[6] - bf_lo(hi4.w), h[7] - bf_hi(hi4.w));
+        __nv_bfloat16* blob = p.ws_hin + ch_head * 2 * N * P;
+        *reinterpret_cast<uint4*>(blob + ((size_t)g * P + ch) * 8) = hi4;
+        *reinterpret_cast<uint4*>(blob + (size_t)N * P + ((size_t)g * P + ch) * 8) = lo4;
+        const float decay = ex2(__ldg(p.ws_decay + ch_head) * kLog2e);
+        const float4* sp = reinterpret_cast<const float4*>(p.ws_S + (ch_head * P + ch) * N + g * 8);
+        const float4 a = sp[0], b = sp[1];
+        h[0] = fmaf(decay, h[0], a.x); h[1] = fmaf(decay, h[1], a.y); h[2] = fmaf(decay, h[2], a.z); h[3] = fmaf(decay, h[3], a.w);
+        h[4] = fmaf(decay, h[4], b.x); h[5] = fmaf(decay, h[5], b.y); h[6] = fmaf(decay, h[6], b.z); h[7] = fmaf(decay, h[7], b.w);
+    }
+    if (fslot < 0) return;
+    if (nck > 0 || fslot != islot) {
+        float4* dst = reinterpret_cast<float4*>(p.pool.ssm + (size_t)fslot * p.pool.ssm_slot_stride + (size_t)d * N + g * 8);
+        dst[0] = make_float4(h[0], h[1], h[2], h[3]);
+        dst[1] = make_float4(h[4], h[5], h[6], h[7]);
+    }
+    if (nck == 0 && fslot != islot && g == 0) {   // a sequence without tokens: its window moves with its state
+        __nv_bfloat16* dc = static_cast<__nv_bfloat16*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride;
+        const __nv_bfloat16* sc = islot >= 0 ? static_cast<const __nv_bfloat16*>(p.pool.conv) + (size_t)islot * p.pool.conv_slot_stride : nullptr;
+        for (int j = 0; j < kW - 1; ++j) dc[(size_t)j * D + d] = sc ? sc[(size_t)j * D + d] : __float2bfloat16_rn(0.0f);
+    }
+}
+
+// ---------------------------------------------------------------- kernel 3: outputs of a chunk
+struct ScanSmem {
+    __nv_bfloat16 Ct[N / 8][Q][8];                       // C rows: A operand of G and of C H_in^T (K-major)
+    union {
+        __nv_bfloat16 Bt[N / 8][Q][8];                   // B rows: B operand of G (K-major) ...
+        __nv_bfloat16 M[Q / 8][Q][8];                    // ... then the masked G: A operand of Y (K-major over the source token)
+    };
+    unsigned char xd[(P / 8) * kXdColBytes];             // Xd = Delta u: B operand of Y (MN-major)
+    __nv_bfloat16 hin[2][N / 8][P][8];                   // incoming state, bf16 value and bf16 remainder: B operands of C H_in^T (K-major)
+    __nv_bfloat16 xs_ext[(Q + 3) * P];                   // 3 rows before the chunk + the x box
+    __nv_bfloat16 zs[Q * P];                             // the z box
+    float ystage[Q][P + 1];                              // y rows on their way from accumulator lanes to channel-contiguous stores
+    RowScalars rs;
+    uint64_t bar_in, bar_z, bar_g, bar_y;
+    uint32_t tmem_base;
+};
+
+__global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
+    extern __shared__ __align__(1024) unsigned char s_raw[];
+    ScanSmem& sm = *reinterpret_cast<ScanSmem*>(s_raw + ((1024u - (smem_u32(s_raw) & 1023u)) & 1023u));
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads, D = p.L.d_inner;
+    const ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, Q, cidx);
+    if (ci.seq < 0) return;
+    const int islot = load_slot(p.init_slot, ci.seq), fslot = load_slot(p.final_slot, ci.seq);
+    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;
+    const int rows = ci.t1 - ci.t0;
+
+    if (tid == 0) {
+        mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_z, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_y, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(&sm.bar_in, Q * P * 2 + 2 * Q * N * 2 + 2 * N * P * 2);
+        tma_box(sm.xs_ext + 3 * P, &maps.x, head * P, ci.t0, &sm.bar_in);
+#pragma unroll
+        for (int c = 0; c < N / 8; ++c) {
+            tma_box(&sm.Ct[c][0][0], &maps.C, c * 8, ci.t0, &sm.bar_in);
+            tma_box(&sm.Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_in);
+        }
+        bulk_load(&sm.hin[0][0][0][0], p.ws_hin + ((size_t)cidx * H + head) * 2 * N * P, 2 * N * P * 2, &sm.bar_in);
+        mbar_expect_tx(&sm.bar_z, Q * P * 2);
+        tma_box(sm.zs, &maps.z, head * P, ci.t0, &sm.bar_z);
+    }
+    if (warp == 0) { tmem_alloc(&sm.tmem_base, 256); tc_fence_before(); }
+    load_halo(sm.xs_ext, p, ci, head, islot);
+    row_scalars(sm.rs, p, head, ci.t0, rows);
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const uint32_t tG = tmem, tYi = tmem + 128, tYx = tmem + 192;   // accumulator columns: G, Y inside the chunk, C H_in^T
+
+    bool ok = mbar_wait_bounded(&sm.bar_in, 0u);
+    if (ok && tid == 0) {
+        tc_fence_after();
+        const uint32_t c0 = smem_u32(&sm.Ct[0][0][0]), b0 = smem_u32(&sm.Bt[0][0][0]), h0 = smem_u32(&sm.hin[0][0][0][0]);
+        constexpr uint32_t idG = instr_desc(Q, false, false), idX = instr_desc(P, false, false);
+#pragma unroll
+        for (int k = 0; k < N / 16; ++k)   // G[t][s] = sum_n C[t][n] B[s][n]
+            mma_bf16(tG, operand_desc(c0 + k * 2 * kColBytes, kColBytes, 128), operand_desc(b0 + k * 2 * kColBytes, kColBytes, 128), idG, k > 0);
+#pragma unroll
+        for (int k = 0; k < 2 * (N / 16); ++k) {   // Yx[t][p] = sum_n C[t][n] h_in[p][n], value then remainder
+            const int kk = k % (N / 16), part = k / (N / 16);
+            mma_bf16(tYx, operand_desc(c0 + kk * 2 * kColBytes, kColBytes, 128),
+                     operand_desc(h0 + part * (N * P * 2) + kk * 2 * kHinColBytes, kHinColBytes, 128), idX, k > 0);
+        }
+        mma_commit(&sm.bar_g);
+    }
+    // conv + SiLU of the warp's 32 rows; u stays in registers for the epilogue, Delta u goes to the operand buffer
+    float ua[32], ub[32];
+    if (ok) {
+        conv_rows(sm.xs_ext, p.L, head, [&](int r, float a, float b) {
+            ua[r & 31] = a; ub[r & 31] = b;
+            const float dl = r < rows ? sm.rs.delta[r] : 0.0f;
+            const uint32_t v = r < rows ? pack_bf(dl * a, dl * b) : 0u;
+            *reinterpret_cast<uint32_t*>(sm.xd + (uint32_t)(lane >> 2) * kXdColBytes + (uint32_t)r * 16u + (uint32_t)(lane & 3) * 4u) = v;
+        });
+    }
+    bool g_ok = ok && mbar_wait_bounded(&sm.bar_g, 0u);
+    if (g_ok) {
+        tc_fence_after();
+        // row t of G, masked: M[t][s] = G[t][s] exp(cs_t - cs_s) for s <= t, else 0; written over the B boxes (G is complete)
+        const float my = sm.rs.csl[tid];
+#pragma unroll 1
+        for (int cb = 0; cb < Q / 32; ++cb) {
+            uint32_t packed[16];
+            if (cb <= warp) {   // column blocks right of the warp's rows are all zero
+                float g[32];
+                tmem_ld32(tG + ((uint32_t)(warp * 32) << 16) + cb * 32, g);
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    const int s0 = cb * 32 + j;
+                    const float m0 = s0 <= tid ? g[j] * ex2(my - sm.rs.csl[s0]) : 0.0f;
+                    const float m1 = s0 + 1 <= tid ? g[j + 1] * ex2(my - sm.rs.csl[s0 + 1]) : 0.0f;
+                    packed[j >> 1] = pack_bf(m0, m1);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) packed[j] = 0u;
+            }
+#pragma unroll
+            for (int u4 = 0; u4 < 4; ++u4)
+                *reinterpret_cast<uint4*>(&sm.M[cb * 4 + u4][tid][0]) = make_uint4(packed[4 * u4], packed[4 * u4 + 1], packed[4 * u4 + 2], packed[4 * u4 + 3]);
+        }
+    }
+    fence_async_smem();
+    tc_fence_before();
+    const bool all_ok = !__syncthreads_or(!g_ok);
+    if (all_ok && tid == 0) {
+        tc_fence_after();
+        const uint32_t m0 = smem_u32(&sm.M[0][0][0]), x0 = smem_u32(sm.xd);
+        constexpr uint32_t idY = instr_desc(P, false, true);
+#pragma unroll
+        for (int k = 0; k < Q / 16; ++k)   // Yi[t][p] = sum_s M[t][s] Xd[s][p]
+            mma_bf16(tYi, operand_desc(m0 + k * 2 * kColBytes, kColBytes, 128), operand_desc(x0 + k * 256, 128, kXdColBytes), idY, k > 0);
+        mma_commit(&sm.bar_y);
+    }
+    bool y_ok = all_ok && mbar_wait_bounded(&sm.bar_y, 0u);
+    if (y_ok) {
+        tc_fence_after();
+        const float scale = ex2(sm.rs.csl[tid]);   // decay from the chunk's start through row t
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            float yi[32], yx[32];
+            tmem_ld32(tYi + ((uint32_t)(warp * 32) << 16) + half * 32, yi);
+            tmem_ld32(tYx + ((uint32_t)(warp * 32) << 16) + half * 32, yx);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) sm.ystage[tid][half * 32 + j] = fmaf(scale, yx[j], yi[j]);
+        }
+    }
+    y_ok = !__syncthreads_or(!y_ok);
+    const bool z_ok = y_ok && mbar_wait_bounded(&sm.bar_z, 0u);
+    if (z_ok) {
+        // skip term, gate, store: the warp's 32 rows, this lane's channel pair (128 contiguous bytes per row and warp)
+        const int d = head * P + 2 * lane;
+        const float da = p.L.D ? __ldg(p.L.D + d) : 0.0f, db = p.L.D ? __ldg(p.L.D + d + 1) : 0.0f;
+        const uint32_t* zc = reinterpret_cast<const uint32_t*>(sm.zs) + lane;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int r = warp * 32 + i;
+            if (r < rows) {
+                const uint32_t zv = zc[r * (P / 2)];
+                const float oa = fmaf(da, ua[i], sm.ystage[r][2 * lane]) * silu(bf_lo(zv));
+                const float ob = fmaf(db, ub[i], sm.ystage[r][2 * lane + 1]) * silu(bf_hi(zv));
+                *reinterpret_cast<uint32_t*>(p.out + (size_t)(ci.t0 + r) * p.ldo + d) = pack_bf(oa, ob);
+            }
+        }
+        // the sequence's last chunk leaves the window: the last three raw inputs (extended rows rows .. rows + 2)
+        if (ci.k == ci.nck - 1 && fslot >= 0 && warp < 3) {
+            __nv_bfloat16* dc = static_cast<__nv_bfloat16*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride + (size_t)warp * D + d;
+            *reinterpret_cast<uint32_t*>(dc) = reinterpret_cast<const uint32_t*>(sm.xs_ext)[(rows + warp) * (P / 2) + lane];
+        }
+    } else if (tid == 0) {
+        flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
+        if (!ok) mbar_wait_bounded(&sm.bar_in, 0u);
+        mbar_wait_bounded(&sm.bar_z, 0u);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_free(tmem, 256);
+}
+
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+cudaError_t launch_ssd_prefill(const SsdPrefillArgs& p, const SsdMaps& maps, cudaStream_t st) {
+    const int H = p.L.n_heads;
+    cudaError_t e;
+    constexpr size_t smem1 = sizeof(StateSmem) + 1024, smem3 = sizeof(ScanSmem) + 1024;
+    if ((e = allow_smem(ssd_chunk_state_kernel, smem1)) != cudaSuccess) return e;
+    if ((e = allow_smem(ssd_chunk_scan_kernel, smem3)) != cudaSuccess) return e;
+    dim3 grid(H, p.n_chunks_bound);
+    ssd_chunk_state_kernel<<<grid, kThreads, smem1, st>>>(p, maps);
+    dim3 g2((p.L.d_inner * (N / 8) + 255) / 256, p.n_seq);
+    ssd_state_passing_kernel<<<g2, 256, 0, st>>>(p);
+    ssd_chunk_scan_kernel<<<grid, kThreads, smem3, st>>>(p, maps);
+    return cudaGetLastError();
+}
+
+}  // namespace mdraft

@@ -37,3 +37,8 @@ def upload_layer(p, act: str, flags: int = mb.MDRAFT_DT_SOFTPLUS, device="cuda")
 
 def i32(values, device="cuda") -> torch.Tensor:
     return torch.tensor(np.asarray(values, dtype=np.int32), dtype=torch.int32, device=device)
+
+
+def upload_ssd_layer(p, flags: int = mb.MDRAFT_DT_SOFTPLUS, device="cuda") -> mb.SsdLayer:
+    f = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
+    return mb.SsdLayer(f(p.A), f(p.D), f(p.conv_w), f(p.conv_b), f(p.dt_bias), p.headdim, p.d_state, flags)
