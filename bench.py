@@ -463,6 +463,7 @@ def run_ours(args):
                 "fp32_issue_frac_70_ops": 70 * units / (ms * 1e-3) / (SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6),
                 "buffers": n_buf, "launches_per_layer": 3}
 
+    peak_hbm = load_peaks()[0]
     prefill_shapes = None
     if not args.quick:
         cfg4_lens = [int(v) for v in np.diff(gen.seq_lengths(gen.get_config(4)))]
@@ -474,6 +475,66 @@ def run_ours(args):
             "fp32_activations_2048": prefill_leg("f32", [2048], 8, 10),
             "bf16_activations_2048_device_inputs": prefill_leg("bf16", [2048], 8, 10),
         }
+
+    # ---- Mamba-2 (SSD) layer of the same size (24 heads of 64 channels, 128 states): context encode on the tensor cores
+    # and the draft-tree step (memory-bound update of 786 KB states).  Inputs from the SSD recipe (host, seeded).
+    roofline_ssd = None
+    if not args.quick:
+        from paper_2506_01206_b200.device_inputs import upload_ssd_layer
+        SP, SN, NLs = 64, 128, 8
+        scfg = gen.Config(97, "ssd-bench", NLs, D, SN, 4, "bf16", 1, (T, T), "none", 0, rank)
+        s_lays = [upload_ssd_layer(gen.ssd_params(scfg, l, SP, SN), md.MDRAFT_DT_SOFTPLUS, dev) for l in range(NLs)]
+        s_in = [[to_device(a, tdt).to(dev) for a in gen.ssd_inputs(scfg, l, 0, 0, T, SP, SN)] for l in range(NLs)]
+        s_out = [torch.empty((T, D), dtype=tdt, device=dev) for _ in range(NLs)]
+        s_nodes = 1 + M
+        s_cache = md.StateCache(NLs, s_nodes, D, d_state=SN, act=tdt, device=dev)
+        s_ws = torch.empty(md.mdraft_ssd_prefill_workspace_bytes(s_lays[0], T, 1), dtype=torch.uint8, device=dev)
+        s_status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+        def ssd_prefill():
+            for l in range(NLs):
+                md.mdraft_ssd_prefill(s_lays[l], s_cache, l, *s_in[l], s_out[l], None, None, slot0, s_ws, s_status)
+
+        s_nin = [[to_device(a, tdt).to(dev) for a in gen.ssd_inputs(scfg, l, 0, 1, M, SP, SN)] for l in range(NLs)]
+        s_nout = [torch.empty((M, D), dtype=tdt, device=dev) for _ in range(NLs)]
+
+        def ssd_tree():
+            for l in range(NLs):
+                md.mdraft_ssd_tree_step(s_lays[l], s_cache, l, *s_nin[l], s_nout[l], parent_slot, node_slot, levels, s_status)
+
+        ms_sp = time_graph(capture(ssd_prefill), Kp, 3) / NLs
+        ms_st = time_graph(capture(ssd_tree), Kp, 3) / NLs
+        if int(s_status.item()):
+            raise RuntimeError("device status bits set in the SSD leg")
+        Hh = D // SP
+        sp_bytes = 3 * T * D * 2 + T * Hh * 2 + 2 * T * SN * 2 + D * SN * 4 + 3 * D * 2
+        n_chunks = -(-T // 128)
+        # tensor-core work as issued: per (chunk, head) G 128x128x128, Y 128x64x128, C.H_in 128x64x128 twice (value and
+        # remainder), state 128x64x128 twice; algorithmic: G once per chunk, no remainder products
+        flops_issued = n_chunks * Hh * 2 * 128 * (128 * 128 + 64 * 128 + 2 * 64 * 128 + 2 * 64 * 128)
+        flops_alg = n_chunks * 2 * 128 * 128 * 128 + n_chunks * Hh * 2 * 128 * (64 * 128 + 64 * 128 + 64 * 128)
+        state_b = D * SN * 4 + 3 * D * 2
+        st_bytes = M * (state_b + 2 * D * 2 + Hh * 2 + D * 2 + 2 * SN * 2) + len(set(int(v) for v in w.tree.parents)) * state_b
+        try:
+            tf_peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+        except Exception:
+            tf_peak = 1590.0
+        roofline_ssd = {
+            "workload": "Mamba-2 (SSD) layer: %d tokens x %d channels = %d heads x 64, 128 states, bf16; %d distinct layers per replay" % (T, D, Hh, NLs),
+            "prefill": {"bound": "hbm", "kernels": "ssd_chunk_state (tcgen05) + ssd_state_passing + ssd_chunk_scan (tcgen05)",
+                        "us_per_layer": ms_sp * 1e3, "algorithmic_bytes_per_layer": sp_bytes,
+                        "achieved": sp_bytes / (ms_sp * 1e-3) / 1e9, "peak": peak_hbm, "unit": "GB/s", "frac": sp_bytes / (ms_sp * 1e-3) / 1e9 / peak_hbm,
+                        "tensor": {"issued_tflops": flops_issued / (ms_sp * 1e-3) / 1e12, "algorithmic_tflops": flops_alg / (ms_sp * 1e-3) / 1e12,
+                                   "peak": tf_peak, "frac_issued": flops_issued / (ms_sp * 1e-3) / 1e12 / tf_peak},
+                        "token_channels_per_s": T * D / (ms_sp * 1e-3),
+                        "note": "HBM binds before the tensor cores at this shape (20.8 MB against 2.9 GFLOP per layer); the kernels are "
+                                "far from either: one 256-thread block per SM walks its phases one after another"},
+            "tree_step": {"bound": "hbm", "kernel": "ssd_step_kernel", "nodes": M, "levels": len(levels) - 1, "us_per_layer_round": ms_st * 1e3,
+                          "algorithmic_bytes_per_layer_round": st_bytes, "achieved": st_bytes / (ms_st * 1e-3) / 1e9, "peak": peak_hbm, "unit": "GB/s",
+                          "frac": st_bytes / (ms_st * 1e-3) / 1e9 / peak_hbm, "node_updates_per_s": M / (ms_st * 1e-3)},
+        }
+        del s_in, s_out, s_cache, s_nin, s_nout
+        torch.cuda.empty_cache()
     clocks = sampler.stop()
 
     # ---- end to end: pinned host inputs -> device -> the path -> outputs back to the host, every step, through the
@@ -669,6 +730,7 @@ def run_ours(args):
             "phases": extra,
             "general_A": general,
             "prefill_shapes": prefill_shapes,
+            "roofline_ssd": roofline_ssd,
             "projection_level": proj_level,
             "drafter_round": drafter,
             "cpu_baseline": cpu,

@@ -32,7 +32,8 @@ namespace mdraft {
 namespace {
 
 constexpr int P = kSsdP, N = kSsdN, Q = kSsdQ;
-constexpr int kThreads = 128;                 // one thread per chunk row / accumulator lane
+constexpr int kThreads = 256;                 // two warps per 32 accumulator lanes: warps w and w + 4 share rows 32 (w % 4) .. and split the columns
+constexpr int kRowsPerWarp = Q / (kThreads / 32);   // rows of the chunk a warp convolves and stores
 constexpr uint32_t kColBytes = Q * 16;        // one 8-wide column of core matrices over 128 rows: 2048 bytes
 constexpr uint32_t kXdColBytes = Q * 16 + 16; // the same for the thread-written Xd / Xw operand, padded against bank conflicts
 constexpr uint32_t kHinColBytes = P * 16;     // H_in: 64 rows
@@ -134,8 +135,9 @@ struct RowScalars {
 
 __device__ __forceinline__ void row_scalars(RowScalars& rs, const SsdPrefillArgs& p, int head, int t0, int rows) {
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const bool owner = t < Q;   // threads Q.. only take part in the barriers
     float delta = 0.0f;
-    if (t < rows) {
+    if (owner && t < rows) {
         const float v = __bfloat162float(p.dt[(size_t)(t0 + t) * p.lddt + head]) + (p.L.dt_bias ? __ldg(p.L.dt_bias + head) : 0.0f);
         delta = (p.L.flags & MDRAFT_DT_SOFTPLUS) ? softplus(v) : v;
     }
@@ -146,14 +148,16 @@ __device__ __forceinline__ void row_scalars(RowScalars& rs, const SsdPrefillArgs
         const float up = __shfl_up_sync(0xffffffffu, la, o);
         if (lane >= o) la += up;
     }
-    if (lane == 31) rs.warp_sum[warp] = la;
+    if (owner && lane == 31) rs.warp_sum[warp] = la;
     __syncthreads();
-    float before = 0.0f;
-    for (int w = 0; w < warp; ++w) before += rs.warp_sum[w];
-    la += before;
-    rs.delta[t] = delta;
-    rs.cs[t] = la;
-    rs.csl[t] = la * kLog2e;
+    if (owner) {
+        float before = 0.0f;
+        for (int w = 0; w < warp; ++w) before += rs.warp_sum[w];
+        la += before;
+        rs.delta[t] = delta;
+        rs.cs[t] = la;
+        rs.csl[t] = la * kLog2e;
+    }
     __syncthreads();
 }
 
@@ -170,7 +174,7 @@ __device__ __forceinline__ void load_halo(__nv_bfloat16* xs_ext, const SsdPrefil
     *reinterpret_cast<uint32_t*>(xs_ext + j * P + 2 * lane) = v;
 }
 
-// conv + SiLU of the warp's 32 rows for this lane's channel pair; calls f(row, u_lo, u_hi) for every row.
+// conv + SiLU of the warp's kRowsPerWarp rows for this lane's channel pair; calls f(row, index in the warp, u_lo, u_hi).
 template <typename F>
 __device__ __forceinline__ void conv_rows(const __nv_bfloat16* xs_ext, const SsdLayerDev& L, int head, F&& f) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -179,17 +183,17 @@ __device__ __forceinline__ void conv_rows(const __nv_bfloat16* xs_ext, const Ssd
     const float4 wb = __ldg(reinterpret_cast<const float4*>(L.conv_w + (size_t)(d + 1) * kW));
     const float ba = L.conv_b ? __ldg(L.conv_b + d) : 0.0f, bb = L.conv_b ? __ldg(L.conv_b + d + 1) : 0.0f;
     const uint32_t* col = reinterpret_cast<const uint32_t*>(xs_ext) + lane;   // row r of the chunk is extended row r + 3
-    const int r0 = warp * 32;
+    const int r0 = warp * kRowsPerWarp;
     uint32_t w0 = col[(r0 + 0) * (P / 2)], w1 = col[(r0 + 1) * (P / 2)], w2 = col[(r0 + 2) * (P / 2)];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
+    for (int i = 0; i < kRowsPerWarp; ++i) {
         const uint32_t xv = col[(r0 + i + 3) * (P / 2)];
         float a = fmaf(wa.x, bf_lo(w0), ba), b = fmaf(wb.x, bf_hi(w0), bb);
         a = fmaf(wa.y, bf_lo(w1), a); b = fmaf(wb.y, bf_hi(w1), b);
         a = fmaf(wa.z, bf_lo(w2), a); b = fmaf(wb.z, bf_hi(w2), b);
         a = fmaf(wa.w, bf_lo(xv), a); b = fmaf(wb.w, bf_hi(xv), b);
         w0 = w1; w1 = w2; w2 = xv;
-        f(r0 + i, silu(a), silu(b));
+        f(r0 + i, i, silu(a), silu(b));
     }
 }
 
@@ -233,7 +237,7 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPref
     bool ok = mbar_wait_bounded(&sm.bar_tma, 0u);
     if (ok) {
         const float cs_end_l = sm.rs.csl[Q - 1];
-        conv_rows(sm.xs_ext, p.L, head, [&](int r, float ua, float ub) {
+        conv_rows(sm.xs_ext, p.L, head, [&](int r, int, float ua, float ub) {
             const float wgt = r < rows ? sm.rs.delta[r] * ex2(cs_end_l - sm.rs.csl[r]) : 0.0f;
             const float va = r < rows ? wgt * ua : 0.0f, vb = r < rows ? wgt * ub : 0.0f;
             const uint32_t hi = pack_bf(va, vb);
@@ -261,12 +265,13 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPref
     bool done = all_ok && mbar_wait_bounded(&sm.bar_mma, 0u);
     if (done) {
         tc_fence_after();
-        // thread n holds row n of S^T: 64 values, one per channel of the head; stores are contiguous across threads
-        float* dst = p.ws_S + ((size_t)cidx * H + head) * P * N + tid;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        // a thread holds half a row of S^T (state n = its accumulator lane): 32 of the head's channels; stores are
+        // contiguous across the threads of a warp
+        const int n = (warp & 3) * 32 + lane, half = warp >> 2;
+        float* dst = p.ws_S + ((size_t)cidx * H + head) * P * N + n;
+        {
             float v[32];
-            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + half * 32, v);
+            tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + half * 32, v);
 #pragma unroll
             for (int j = 0; j < 32; ++j) dst[(size_t)(half * 32 + j) * N] = v[j];
         }
@@ -309,21 +314,38 @@ __global__ void __launch_bounds__(256) ssd_state_passing_kernel(const SsdPrefill
         const float4 a = src[0], b = src[1];
         h[0] = a.x; h[1] = a.y; h[2] = a.z; h[3] = a.w; h[4] = b.x; h[5] = b.y; h[6] = b.z; h[7] = b.w;
     }
-    for (int c = first; c < first + nck; ++c) {
-        const size_t ch_head = (size_t)c * H + head;
-        // bf16 value and bf16 remainder of the incoming state: two operands, so that the product with C sees ~16 mantissa bits
-        uint4 hi4, lo4;
-        hi4.x = pack_bf(h[0], h[1]); hi4.y = pack_bf(h[2], h[3]); hi4.z = pack_bf(h[4], h[5]); hi4.w = pack_bf(h[6], h[7]);
-        lo4.x = pack_bf(h[0] - bf_lo(hi4.x), h[1] - bf_hi(hi4.x)); lo4.y = pack_bf(h[2] - bf_lo(hi4.y), h[3] - bf_hi(hi4.y));
-        lo4.z = pack_bf(h[4] - bf_lo(hi4.z), h[5] - bf_hi(hi4.z)); lo4.w = pack_bf(h[6] - bf_lo(hi4.w), h[7] - bf_hi(hi4.w));
-        __nv_bfloat16* blob = p.ws_hin + ch_head * 2 * N * P;
-        *reinterpret_cast<uint4*>(blob + ((size_t)g * P + ch) * 8) = hi4;
-        *reinterpret_cast<uint4*>(blob + (size_t)N * P + ((size_t)g * P + ch) * 8) = lo4;
-        const float decay = ex2(__ldg(p.ws_decay + ch_head) * kLog2e);
-        const float4* sp = reinterpret_cast<const float4*>(p.ws_S + (ch_head * P + ch) * N + g * 8);
-        const float4 a = sp[0], b = sp[1];
-        h[0] = fmaf(decay, h[0], a.x); h[1] = fmaf(decay, h[1], a.y); h[2] = fmaf(decay, h[2], a.z); h[3] = fmaf(decay, h[3], a.w);
-        h[4] = fmaf(decay, h[4], b.x); h[5] = fmaf(decay, h[5], b.y); h[6] = fmaf(decay, h[6], b.z); h[7] = fmaf(decay, h[7], b.w);
+    // Four chunks per round: their summaries are fetched together (the loads do not depend on the running state), then
+    // the state walks through them.
+    const int end = first + nck;
+    for (int c0 = first; c0 < end; c0 += 4) {
+        float4 sa[4], sb[4];
+        float decay[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (c0 + i < end) {
+                const size_t ch_head = (size_t)(c0 + i) * H + head;
+                const float4* sp = reinterpret_cast<const float4*>(p.ws_S + (ch_head * P + ch) * N + g * 8);
+                sa[i] = sp[0]; sb[i] = sp[1];
+                decay[i] = __ldg(p.ws_decay + ch_head);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (c0 + i < end) {
+                const size_t ch_head = (size_t)(c0 + i) * H + head;
+                // bf16 value and bf16 remainder of the incoming state: two operands, so that the product with C sees ~16 mantissa bits
+                uint4 hi4, lo4;
+                hi4.x = pack_bf(h[0], h[1]); hi4.y = pack_bf(h[2], h[3]); hi4.z = pack_bf(h[4], h[5]); hi4.w = pack_bf(h[6], h[7]);
+                lo4.x = pack_bf(h[0] - bf_lo(hi4.x), h[1] - bf_hi(hi4.x)); lo4.y = pack_bf(h[2] - bf_lo(hi4.y), h[3] - bf_hi(hi4.y));
+                lo4.z = pack_bf(h[4] - bf_lo(hi4.z), h[5] - bf_hi(hi4.z)); lo4.w = pack_bf(h[6] - bf_lo(hi4.w), h[7] - bf_hi(hi4.w));
+                __nv_bfloat16* blob = p.ws_hin + ch_head * 2 * N * P;
+                *reinterpret_cast<uint4*>(blob + ((size_t)g * P + ch) * 8) = hi4;
+                *reinterpret_cast<uint4*>(blob + (size_t)N * P + ((size_t)g * P + ch) * 8) = lo4;
+                const float dk = ex2(decay[i] * kLog2e);
+                h[0] = fmaf(dk, h[0], sa[i].x); h[1] = fmaf(dk, h[1], sa[i].y); h[2] = fmaf(dk, h[2], sa[i].z); h[3] = fmaf(dk, h[3], sa[i].w);
+                h[4] = fmaf(dk, h[4], sb[i].x); h[5] = fmaf(dk, h[5], sb[i].y); h[6] = fmaf(dk, h[6], sb[i].z); h[7] = fmaf(dk, h[7], sb[i].w);
+            }
+        }
     }
     if (fslot < 0) return;
     if (nck > 0 || fslot != islot) {
@@ -404,10 +426,10 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefi
         mma_commit(&sm.bar_g);
     }
     // conv + SiLU of the warp's 32 rows; u stays in registers for the epilogue, Delta u goes to the operand buffer
-    float ua[32], ub[32];
+    float ua[kRowsPerWarp], ub[kRowsPerWarp];
     if (ok) {
-        conv_rows(sm.xs_ext, p.L, head, [&](int r, float a, float b) {
-            ua[r & 31] = a; ub[r & 31] = b;
+        conv_rows(sm.xs_ext, p.L, head, [&](int r, int i, float a, float b) {
+            ua[i] = a; ub[i] = b;
             const float dl = r < rows ? sm.rs.delta[r] : 0.0f;
             const uint32_t v = r < rows ? pack_bf(dl * a, dl * b) : 0u;
             *reinterpret_cast<uint32_t*>(sm.xd + (uint32_t)(lane >> 2) * kXdColBytes + (uint32_t)r * 16u + (uint32_t)(lane & 3) * 4u) = v;
@@ -417,18 +439,22 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefi
     if (g_ok) {
         tc_fence_after();
         // row t of G, masked: M[t][s] = G[t][s] exp(cs_t - cs_s) for s <= t, else 0; written over the B boxes (G is complete)
-        const float my = sm.rs.csl[tid];
+        // warps w and w + 4 own rows 32 (w % 4) ..: the first takes column blocks 0 and 3, the second 1 and 2 (five
+        // non-zero blocks of 32 x 32 on each side of the split)
+        const int rb = warp & 3, row = rb * 32 + lane;
+        const float my = sm.rs.csl[row];
 #pragma unroll 1
-        for (int cb = 0; cb < Q / 32; ++cb) {
+        for (int q = 0; q < 2; ++q) {
+            const int cb = warp < 4 ? (q == 0 ? 0 : 3) : (q == 0 ? 1 : 2);
             uint32_t packed[16];
-            if (cb <= warp) {   // column blocks right of the warp's rows are all zero
+            if (cb <= rb) {   // column blocks right of the warp's rows are all zero
                 float g[32];
-                tmem_ld32(tG + ((uint32_t)(warp * 32) << 16) + cb * 32, g);
+                tmem_ld32(tG + ((uint32_t)(rb * 32) << 16) + cb * 32, g);
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
                     const int s0 = cb * 32 + j;
-                    const float m0 = s0 <= tid ? g[j] * ex2(my - sm.rs.csl[s0]) : 0.0f;
-                    const float m1 = s0 + 1 <= tid ? g[j + 1] * ex2(my - sm.rs.csl[s0 + 1]) : 0.0f;
+                    const float m0 = s0 <= row ? g[j] * ex2(my - sm.rs.csl[s0]) : 0.0f;
+                    const float m1 = s0 + 1 <= row ? g[j + 1] * ex2(my - sm.rs.csl[s0 + 1]) : 0.0f;
                     packed[j >> 1] = pack_bf(m0, m1);
                 }
             } else {
@@ -437,7 +463,7 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefi
             }
 #pragma unroll
             for (int u4 = 0; u4 < 4; ++u4)
-                *reinterpret_cast<uint4*>(&sm.M[cb * 4 + u4][tid][0]) = make_uint4(packed[4 * u4], packed[4 * u4 + 1], packed[4 * u4 + 2], packed[4 * u4 + 3]);
+                *reinterpret_cast<uint4*>(&sm.M[cb * 4 + u4][row][0]) = make_uint4(packed[4 * u4], packed[4 * u4 + 1], packed[4 * u4 + 2], packed[4 * u4 + 3]);
         }
     }
     fence_async_smem();
@@ -455,26 +481,24 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefi
     bool y_ok = all_ok && mbar_wait_bounded(&sm.bar_y, 0u);
     if (y_ok) {
         tc_fence_after();
-        const float scale = ex2(sm.rs.csl[tid]);   // decay from the chunk's start through row t
+        const int rb = warp & 3, row = rb * 32 + lane, half = warp >> 2;
+        const float scale = ex2(sm.rs.csl[row]);   // decay from the chunk's start through this row
+        float yi[32], yx[32];
+        tmem_ld32(tYi + ((uint32_t)(rb * 32) << 16) + half * 32, yi);
+        tmem_ld32(tYx + ((uint32_t)(rb * 32) << 16) + half * 32, yx);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            float yi[32], yx[32];
-            tmem_ld32(tYi + ((uint32_t)(warp * 32) << 16) + half * 32, yi);
-            tmem_ld32(tYx + ((uint32_t)(warp * 32) << 16) + half * 32, yx);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) sm.ystage[tid][half * 32 + j] = fmaf(scale, yx[j], yi[j]);
-        }
+        for (int j = 0; j < 32; ++j) sm.ystage[row][half * 32 + j] = fmaf(scale, yx[j], yi[j]);
     }
     y_ok = !__syncthreads_or(!y_ok);
     const bool z_ok = y_ok && mbar_wait_bounded(&sm.bar_z, 0u);
     if (z_ok) {
-        // skip term, gate, store: the warp's 32 rows, this lane's channel pair (128 contiguous bytes per row and warp)
+        // skip term, gate, store: the warp's rows, this lane's channel pair (128 contiguous bytes per row and warp)
         const int d = head * P + 2 * lane;
         const float da = p.L.D ? __ldg(p.L.D + d) : 0.0f, db = p.L.D ? __ldg(p.L.D + d + 1) : 0.0f;
         const uint32_t* zc = reinterpret_cast<const uint32_t*>(sm.zs) + lane;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const int r = warp * 32 + i;
+        for (int i = 0; i < kRowsPerWarp; ++i) {
+            const int r = warp * kRowsPerWarp + i;
             if (r < rows) {
                 const uint32_t zv = zc[r * (P / 2)];
                 const float oa = fmaf(da, ua[i], sm.ystage[r][2 * lane]) * silu(bf_lo(zv));

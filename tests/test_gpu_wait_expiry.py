@@ -122,3 +122,34 @@ def test_projection_step_wait_runs_out_and_the_cluster_still_meets(waitlib, act,
     o_out, _, o_h, _, _, _ = rig.oracle()
     assert_close(out.float().cpu().numpy(), o_out, TOL[act], "node outputs after recovery")
     assert_close(rig.states()[0], o_h, TOL_STATE, "node states after recovery")
+
+
+def test_ssd_prefill_wait_runs_out_tensor_memory_is_freed_and_the_next_call_is_correct(waitlib):
+    """The tensor-core kernels of the SSD encode allocate tensor memory before they wait for their copies: when the
+    wait runs out they must still free it (a leak would stall later blocks on the same SM for good) and store no
+    output.  Several rounds of failing calls, then an ordinary call checked against the oracle."""
+    import oracle
+    from paper_2506_01206_b200.device_inputs import upload_ssd_layer
+    Dn, T, Pn, Nn = 192, 300, 64, 128
+    cfg = gen.Config(95, "ssd-wait", 1, Dn, Nn, 4, "bf16", 1, (1, 1), "none", 0, 0)
+    prm = gen.ssd_params(cfg, 0, Pn, Nn, conv_bias=True)
+    arrs = gen.ssd_inputs(cfg, 0, 0, 0, T, Pn, Nn)
+    lay = upload_ssd_layer(prm)
+    dev = [to_device(a, torch.bfloat16) for a in arrs]
+    cache = md.StateCache(1, 1, Dn, d_state=Nn, act=torch.bfloat16)
+    ws = torch.empty(md.mdraft_ssd_prefill_workspace_bytes(lay, T, 1), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.full((T, Dn), 7.0, dtype=torch.bfloat16, device="cuda")
+    with using(waitlib):
+        for _ in range(6):   # more failing blocks than an SM has tensor-memory columns for, if any were leaked
+            md.mdraft_ssd_prefill(lay, cache, 0, *dev, out, None, None, i32([0]), ws, status)
+        torch.cuda.synchronize()
+    assert int(status.item()) == md.MDRAFT_DEV_WAIT_EXPIRED
+    assert bool((out == 7.0).all()), "a block that gave up must not have written outputs"
+    status.zero_()
+    md.mdraft_ssd_prefill(lay, cache, 0, *dev, out, None, None, i32([0]), ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o_out, _, o_h = oracle.ssd_prefill(oracle.ssd_layer_from_params(prm), *arrs)
+    assert_close(out.float().cpu().numpy(), o_out, TOL["bf16"], "out after recovery")
+    assert_close(cache.ssm[0].cpu().numpy(), o_h, TOL_STATE, "state after recovery")
