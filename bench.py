@@ -427,6 +427,34 @@ def run_ours(args):
                   "projection_step": time_graph(capture(pj_fused), Kp, 3) / NL * 1e3,
                   "split_mode": time_graph(capture(pj_split), Kp, 3) / NL * 1e3,
                   "plain_step_inputs_given": time_graph(capture(pj_plain), Kp, 3) / NL * 1e3}
+    # wide levels: the projection step against the split mode, and what a caller following the header's width rule gets
+    # (projection step up to MDRAFT_PROJ_STEP_MAX_NODES nodes per level, split mode beyond); 8 layers per replay
+    if not args.quick:
+        from paper_2506_01206_b200.drafter import PROJ_STEP_MAX_NODES
+        NLw = 8
+        wide = {}
+        for PNw in (256, 442, 512, 1024):
+            w_in = [[a[:PNw] for a in bt_in[l]] for l in range(NLw)]
+            w_out, w_u = torch.empty((PNw, D), dtype=tdt, device=dev), torch.empty((PNw, D), dtype=tdt, device=dev)
+            w_par, w_nod = i32([0] * PNw, dev), i32(list(range(1, PNw + 1)), dev)
+
+            def w_fused():
+                for l in range(NLw):
+                    md.mdraft_tree_step_proj(bt_layers[l], bt_cache, l, pj_W[l][0], pj_W[l][1], w_in[l][0], w_in[l][1], w_out, w_par, w_nod, bt_status)
+
+            def w_split():
+                for l in range(NLw):
+                    md.mdraft_tree_step(bt_layers[l], bt_cache, l, w_in[l][0], None, None, None, None, w_u, w_par, w_nod, None, bt_status,
+                                        flags=md.MDRAFT_CONV_ONLY)
+                    s_ = w_u @ pj_Wt[l][0]
+                    dt_ = (s_[:, :PR] @ pj_Wt[l][1]).contiguous()
+                    md.mdraft_tree_step(bt_layers[l], bt_cache, l, w_u, w_in[l][1], dt_, s_[:, PR:PR + 16].contiguous(), s_[:, PR + 16:].contiguous(),
+                                        w_out, w_par, w_nod, None, bt_status, flags=fl | md.MDRAFT_PRECONV)
+
+            tf_, ts_ = time_graph(capture(w_fused), Kp, 3) / NLw * 1e3, time_graph(capture(w_split), Kp, 3) / NLw * 1e3
+            wide[str(PNw)] = {"projection_step": tf_, "split_mode": ts_, "by_width_rule": tf_ if PNw <= PROJ_STEP_MAX_NODES else ts_}
+        proj_level["wide_levels_us_per_layer"] = wide
+        proj_level["width_rule"] = "projection step up to %d nodes per level, split mode beyond (include/mdraft.h, drafter.PROJ_STEP_MAX_NODES)" % PROJ_STEP_MAX_NODES
     if int(bt_status.item()):
         raise RuntimeError("device status bits set in the projection leg")
 

@@ -246,7 +246,15 @@ int mdraft_tree_step(const mdraft_layer *layer, const mdraft_cache *cache, int32
  * MDRAFT_CONV_ONLY make no sense here (MDRAFT_ERR_INVALID_ARG).  d_inner above 4096 is
  * MDRAFT_ERR_UNSUPPORTED (the blocks of a node must fit one cluster): use the split mode there.
  * Device-side faults are reported through dev_status as in mdraft_tree_step.
+ *
+ * Width of a level.  The call is built for the level widths of drafting (the paper's trees have 1 to 18 nodes per
+ * level; it is about twice as fast as the split mode there).  Every node's blocks read both matrices again (out of
+ * L2), so the cost per node does not fall with the width, while the split mode's matrix products amortise the weights
+ * over the level: beyond MDRAFT_PROJ_STEP_MAX_NODES nodes per level the split mode (MDRAFT_CONV_ONLY step, the
+ * caller's two matrix products, MDRAFT_PRECONV step) is the faster path and callers should switch to it there, as
+ * the package's block stack does.  The call itself accepts any width and stays correct.
  */
+#define MDRAFT_PROJ_STEP_MAX_NODES 256
 typedef struct mdraft_select_proj {
     const void *W_x;
     const void *W_dt;

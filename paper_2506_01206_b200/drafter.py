@@ -24,6 +24,11 @@ import torch
 from . import binding as mb
 
 
+# Above this many nodes in a level the one-launch projection step loses to the split mode (its per-node re-reads of
+# the two projection matrices cost more than the split mode's matrix products); the stack switches path there.
+PROJ_STEP_MAX_NODES = 256
+
+
 class ToyDrafter:
     def __init__(self, n_layers: int = 24, d_model: int = 768, d_inner: int = 1536, dt_rank: int = 48, vocab: int = 50280,
                  max_nodes: int = 64, act: torch.dtype = torch.bfloat16, seed: int = 0, device="cuda", fused: bool = False):
@@ -78,7 +83,7 @@ class ToyDrafter:
         for l in range(self.n_layers):
             xz = self._norm(h) @ self.W_in[l]
             x, z = xz[:, :self.d_inner], xz[:, self.d_inner:]
-            if self.fused:
+            if self.fused and hi - lo <= PROJ_STEP_MAX_NODES:
                 mb.mdraft_tree_step_proj(self.layers[l], self.cache, l, self.W_x_rows[l], self.W_dt_rows[l], x, z, y, ps, ns, self.status,
                                          flags=mb.MDRAFT_DT_SOFTPLUS | mb.MDRAFT_A_POWERS)
                 h = h + y @ self.W_out[l]

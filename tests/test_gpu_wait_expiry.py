@@ -91,7 +91,7 @@ def test_tree_step_wait_runs_out_and_the_call_returns(waitlib, act):
     tree = gen.paper_tree((3, 2, 2, 1, 1))
     rig = TreeRig(cfg, tree)
     with using(waitlib):
-        out = rig.step(0, tree.n_nodes, level_offsets=[int(v) for v in tree.level_offsets])
+        out = rig.run_levels()   # one call per level: the kernel that stages a node's data with bulk copies
     assert int(rig.status.item()) == md.MDRAFT_DEV_WAIT_EXPIRED
     assert bool(torch.isnan(out).all()), "no node output may have been written"
     assert bool(torch.isnan(rig.cache.ssm[0, 1:]).all()) and bool(torch.isnan(rig.cache.conv[0, 1:].float()).all()), "no node slot either"
