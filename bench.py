@@ -9,7 +9,7 @@ workload (Mamba-130M: 24 layers, d_inner 1536, d_state 16; context 2048 tokens; 
 the per-phase throughputs (prefill token*channels/s, tree node-updates/s) are reported beside it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-    python bench.py --profile-case prefill|tree|proj [sizes ...]     (small runs of one kernel family for a profiler)
+    python bench.py --profile-case prefill|tree|proj|ssd [sizes ...] (small runs of one kernel family for a profiler)
 
 N > 1 (under torchrun) runs N independent replicas (the path has no exchange step): weak scaling.
 `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
@@ -773,7 +773,8 @@ def profile_case(what, sizes):
     inputs larger than L2 across the layers so that DRAM counters still mean something.
       prefill [tokens=2048] [layers=4] [reps=3] [fp32=0]   130M-shaped context encode, bf16 (or fp32) activations, structured A
       tree    [layers=4] [reps=2]                          one batched-serving draft round, 32 sequences x 32-node trees
-      proj    [nodes=18] [layers=24] [reps=3]              one tree level through the step that forms dt, B, C itself"""
+      proj    [nodes=18] [layers=24] [reps=3]              one tree level through the step that forms dt, B, C itself
+      ssd     [tokens=2048] [layers=2] [reps=3]            Mamba-2 (SSD) context encode, 24 heads x 64 channels, 128 states"""
     import torch
     import paper_2506_01206_b200 as md
     from paper_2506_01206_b200.device_inputs import i32, to_device, torch_act, upload_layer
@@ -811,6 +812,23 @@ def profile_case(what, sizes):
                 md.mdraft_tree_step(lays[l], cache, l, *ins[l], outs[l], par, nod, bt.levels, status)
         torch.cuda.synchronize()
         print("tree: %d nodes, levels %s, %d layers x %d, status %d" % (bt.M, np.diff(bt.levels).tolist(), n_layers, reps, int(status.item())))
+    elif what == "ssd":
+        from paper_2506_01206_b200.device_inputs import upload_ssd_layer
+        tokens, n_layers, reps = (list(sizes) + [2048, 2, 3][len(sizes):])[:3]
+        D, P, N = 1536, 64, 128
+        cfg = gen.Config(97, "ssd-profile", n_layers, D, N, 4, "bf16", 1, (tokens, tokens), "none", 0, 0)
+        tdt = torch.bfloat16
+        lays = [upload_ssd_layer(gen.ssd_params(cfg, l, P, N)) for l in range(n_layers)]
+        ins = [[to_device(a, tdt) for a in gen.ssd_inputs(cfg, l, 0, 0, tokens, P, N)] for l in range(n_layers)]
+        outs = [torch.empty((tokens, D), dtype=tdt, device="cuda") for _ in range(n_layers)]
+        cache = md.StateCache(n_layers, 1, D, d_state=N, act=tdt)
+        ws = torch.empty(md.mdraft_ssd_prefill_workspace_bytes(lays[0], tokens, 1), dtype=torch.uint8, device="cuda")
+        slot = i32([0])
+        for _ in range(reps):
+            for l in range(n_layers):
+                md.mdraft_ssd_prefill(lays[l], cache, l, *ins[l], outs[l], None, None, slot, ws, status)
+        torch.cuda.synchronize()
+        print("ssd: %d tokens x %d channels (%d heads), %d layers x %d, status %d" % (tokens, D, D // P, n_layers, reps, int(status.item())))
     else:
         n_nodes, n_layers, reps = (list(sizes) + [18, 24, 3][len(sizes):])[:3]
         dt_rank = 48
@@ -838,7 +856,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--quick", action="store_true", help="skip the further prefill shapes (long context, packed batch, fp32)")
-    ap.add_argument("--profile-case", choices=["prefill", "tree", "proj"], help="run one small kernel case for a profiler and exit")
+    ap.add_argument("--profile-case", choices=["prefill", "tree", "proj", "ssd"], help="run one small kernel case for a profiler and exit")
     ap.add_argument("sizes", nargs="*", type=int, help="sizes of the profile case (see profile_case)")
     args = ap.parse_args()
     if args.profile_case:

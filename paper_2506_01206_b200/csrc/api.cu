@@ -16,7 +16,18 @@ using namespace mdraft;
 
 namespace {
 
-constexpr int kSmCount = 148;  // B200
+constexpr int kSmCountB200 = 148;
+
+// SMs of the current device; the B200's count when no device can be asked (the workspace query also runs where there
+// is none, and must then give the size the call will want on the B200 it is planned for).
+int sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        (void)cudaGetLastError();
+        return kSmCountB200;
+    }
+    return n;
+}
 
 inline size_t elem_size(int act) { return act == MDRAFT_BF16 ? 2 : 4; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -100,7 +111,8 @@ PrefillPlan plan_prefill(const mdraft_layer* L, int T, int n_seq, int max_seqlen
     if (opts && opts->chunk_len > 0) {
         Lc = opts->chunk_len < 4 ? 4 : opts->chunk_len;
     } else {
-        int want = wide ? kSmCount / ch_blocks_wide : kSmCount * kBlocksPerSm / ch_blocks;
+        const int sms = sm_count();
+        int want = wide ? sms / ch_blocks_wide : sms * kBlocksPerSm / ch_blocks;
         if (want < 1) want = 1;
         Lc = (T + want - 1) / want;
         if (Lc < kMinChunk) Lc = kMinChunk;
@@ -410,7 +422,7 @@ SsdLayerDev ssd_layer_dev(const mdraft_ssd_layer* L) {
 
 struct SsdPlan {
     int n_chunks_bound;
-    size_t off_S, off_decay, off_hin, bytes;
+    size_t off_S, off_decay, off_hin, off_xd, off_u, off_csl, bytes;
 };
 
 SsdPlan plan_ssd(const mdraft_ssd_layer* L, int T, int n_seq) {
@@ -421,7 +433,10 @@ SsdPlan plan_ssd(const mdraft_ssd_layer* L, int T, int n_seq) {
     pl.off_S = 0;
     pl.off_decay = align_up(pl.off_S + (size_t)pl.n_chunks_bound * per_chunk * sizeof(float), 256);
     pl.off_hin = align_up(pl.off_decay + (size_t)pl.n_chunks_bound * H * sizeof(float), 256);
-    pl.bytes = align_up(pl.off_hin + (size_t)pl.n_chunks_bound * per_chunk * 2 * 2, 256);   // bf16 value + bf16 remainder
+    pl.off_xd = align_up(pl.off_hin + (size_t)pl.n_chunks_bound * per_chunk * 2 * 2, 256);   // bf16 value + bf16 remainder
+    pl.off_u = align_up(pl.off_xd + (size_t)pl.n_chunks_bound * H * (kSsdP / 8) * (kSsdQ * 16 + 16), 256);
+    pl.off_csl = align_up(pl.off_u + (size_t)T * L->d_inner * 2, 256);
+    pl.bytes = align_up(pl.off_csl + (size_t)pl.n_chunks_bound * H * kSsdQ * sizeof(float), 256);
     return pl;
 }
 
@@ -486,6 +501,9 @@ int mdraft_ssd_prefill(const mdraft_ssd_layer* layer, const mdraft_cache* cache,
     a.ws_S = reinterpret_cast<float*>(ws + pl.off_S);
     a.ws_decay = reinterpret_cast<float*>(ws + pl.off_decay);
     a.ws_hin = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_hin);
+    a.ws_xd = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_xd);
+    a.ws_u = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_u);
+    a.ws_csl = reinterpret_cast<float*>(ws + pl.off_csl);
     a.dev_status = dev_status;
     SsdMaps maps;
     memset(&maps, 0, sizeof(maps));

@@ -40,6 +40,9 @@ struct SsdPrefillArgs {
     float* ws_S;               // [chunk][H][P][N] fp32: what the chunk adds to a zero state
     float* ws_decay;           // [chunk][H]       fp32: sum over the chunk of Delta * A (log of the chunk's decay)
     __nv_bfloat16* ws_hin;     // [chunk][H][2][N/8][P][8] bf16: the chunk's incoming state (value, remainder), laid out as the tensor-core operand
+    __nv_bfloat16* ws_xd;      // [chunk][H][P/8][Q (+1 unit of padding)][8] bf16: Delta * u in operand layout (kernel 1 -> kernel 3)
+    __nv_bfloat16* ws_u;       // [T][D] bf16: conv + SiLU output, for the skip term (kernel 1 -> kernel 3)
+    float* ws_csl;             // [chunk][H][Q] fp32: running log2-decay of the chunk's rows (kernel 1 -> kernel 3)
     int32_t* dev_status;
 };
 

@@ -9,13 +9,16 @@
 //     h_out = exp(cs_end) h_in + S
 //
 // Three stream-ordered kernels, none waiting on another block:
-//   1. ssd_chunk_state: per (head, chunk) S^T = B^T Xw on the tensor cores (tcgen05.mma, bf16 operands, fp32 accumulator
-//      in tensor memory); Xw is split into a bf16 value and a bf16 remainder (two products into one accumulator) so that
-//      the state keeps fp32-level accuracy.
+//   1. ssd_chunk_state: per (head, chunk) conv + SiLU, step sizes and running decays, then S^T = B^T Xw on the tensor
+//      cores (tcgen05.mma, bf16 operands, fp32 accumulator in tensor memory); Xw is split into a bf16 value and a bf16
+//      remainder (two products into one accumulator) so that the state keeps fp32-level accuracy.  What kernel 3 needs
+//      of this work is handed over through the workspace: Xd = Delta u already in operand layout, u, and the running
+//      log-decays of the chunk's rows; the sequence's last chunk also leaves the conv window.
 //   2. ssd_state_passing: per (channel, 8 states) the chunk states of a sequence are chained in token order; every
 //      chunk's incoming state is left in the operand layout the next kernel wants, the final state goes to its slot.
 //   3. ssd_chunk_scan: per (head, chunk) G = C B^T, the causal decay mask applied to G on its way from tensor memory to
-//      shared memory, Y = (G o L) Xd and C H_in^T on the tensor cores, then skip term, gate and store.
+//      shared memory, Y = (G o L) Xd and C H_in^T on the tensor cores, then skip term, gate and store.  It touches no
+//      x, dt or conv weight: its shared memory is three operand tiles, so that two blocks share an SM.
 //
 // Operands live in shared memory in the tensor core's canonical un-swizzled layout: 16-byte units of 8 bf16 values,
 // 8 units = one 8 x 8 "core matrix" of 128 contiguous bytes; one descriptor field gives the byte step between core
@@ -202,6 +205,7 @@ struct StateSmem {
     __nv_bfloat16 Bt[N / 8][Q][8];                        // B rows of the chunk, one TMA box per 8 states
     unsigned char xw_hi[(P / 8) * kXdColBytes];           // Xw = Delta exp(cs_end - cs) u, bf16 value ...
     unsigned char xw_lo[(P / 8) * kXdColBytes];           // ... and bf16 remainder
+    unsigned char xd[(P / 8) * kXdColBytes];              // Xd = Delta u, the operand of the chunk-scan kernel (sent to the workspace)
     __nv_bfloat16 xs_ext[(Q + 3) * P];                    // 3 rows before the chunk + the x box
     RowScalars rs;
     uint64_t bar_tma, bar_mma;
@@ -245,11 +249,24 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPref
             const uint32_t off = (uint32_t)(lane >> 2) * kXdColBytes + (uint32_t)r * 16u + (uint32_t)(lane & 3) * 4u;
             *reinterpret_cast<uint32_t*>(sm.xw_hi + off) = hi;
             *reinterpret_cast<uint32_t*>(sm.xw_lo + off) = lo;
+            const float dl = r < rows ? sm.rs.delta[r] : 0.0f;
+            *reinterpret_cast<uint32_t*>(sm.xd + off) = r < rows ? pack_bf(dl * ua, dl * ub) : 0u;
+            if (r < rows) *reinterpret_cast<uint32_t*>(p.ws_u + (size_t)(ci.t0 + r) * p.L.d_inner + head * P + 2 * lane) = pack_bf(ua, ub);
         });
+        if (tid < Q) p.ws_csl[((size_t)cidx * H + head) * Q + tid] = sm.rs.csl[tid];
+        // the sequence's last chunk leaves the window: the last three raw inputs (extended rows rows .. rows + 2)
+        if (ci.k == ci.nck - 1 && fslot >= 0 && warp < 3) {
+            __nv_bfloat16* dc = static_cast<__nv_bfloat16*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride + (size_t)warp * p.L.d_inner + head * P + 2 * lane;
+            *reinterpret_cast<uint32_t*>(dc) = reinterpret_cast<const uint32_t*>(sm.xs_ext)[(rows + warp) * (P / 2) + lane];
+        }
     }
-    fence_async_smem();   // the operand written by threads must be visible to the tensor core's reads
+    fence_async_smem();   // the operands written by threads must be visible to the tensor core's and the copy engine's reads
     const bool all_ok = !__syncthreads_or(!ok);
     if (all_ok && tid == 0) {
+        // Xd leaves for the workspace as one bulk store (same bytes, same layout as the chunk-scan kernel's operand)
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(p.ws_xd + ((size_t)cidx * H + head) * (sizeof(sm.xd) / 2))),
+                     "r"(smem_u32(sm.xd)), "r"((uint32_t)sizeof(sm.xd)) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         tc_fence_after();
         // S^T (n x p) = sum over tokens: A operand = B^T read MN-major out of the TMA boxes, B operand = Xw MN-major.
         constexpr uint32_t idesc = instr_desc(P, true, true);
@@ -280,6 +297,7 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPref
         flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
         if (!ok) mbar_wait_bounded(&sm.bar_tma, 0u);   // the copies target this block's shared memory: one more bounded chance
     }
+    if (all_ok && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory stays valid until the store has read it
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_free(tmem, 64);
@@ -288,10 +306,10 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPref
 // ---------------------------------------------------------------- kernel 2: chain the chunk states of a sequence
 // Thread = (channel d, group of 8 states).  Walks the sequence's chunks in order: writes the chunk's incoming state as
 // bf16 (a value and a remainder) in the operand layout [state group][channel of the head][8], then h <- exp(chunk decay) h + S.
-__global__ void __launch_bounds__(256) ssd_state_passing_kernel(const SsdPrefillArgs p) {
+__global__ void __launch_bounds__(128) ssd_state_passing_kernel(const SsdPrefillArgs p) {
     const int D = p.L.d_inner, H = p.L.n_heads;
     const int s = blockIdx.y;
-    const int idx = blockIdx.x * 256 + threadIdx.x;
+    const int idx = blockIdx.x * 128 + threadIdx.x;
     int first, nck;
     seq_chunks(p.cu, p.n_seq, p.T, Q, s, first, nck);   // whole warps call this
     // malformed offsets: the sequence has no chunk and is skipped
@@ -305,7 +323,9 @@ __global__ void __launch_bounds__(256) ssd_state_passing_kernel(const SsdPrefill
         return;
     }
     if (idx >= D * (N / 8)) return;
-    const int g = idx % (N / 8), d = idx / (N / 8), head = d / P, ch = d % P;   // consecutive threads: consecutive state groups of one channel
+    // consecutive threads: consecutive channels of one head and one state group, so that the 16-byte operand words they
+    // write are contiguous (their 32-byte reads of the chunk states each fill a sector of their own)
+    const int ch = idx % P, g = (idx / P) % (N / 8), head = idx / (P * (N / 8)), d = head * P + ch;
     float h[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) h[i] = 0.0f;
@@ -314,14 +334,15 @@ __global__ void __launch_bounds__(256) ssd_state_passing_kernel(const SsdPrefill
         const float4 a = src[0], b = src[1];
         h[0] = a.x; h[1] = a.y; h[2] = a.z; h[3] = a.w; h[4] = b.x; h[5] = b.y; h[6] = b.z; h[7] = b.w;
     }
-    // Four chunks per round: their summaries are fetched together (the loads do not depend on the running state), then
+    // Eight chunks per round: their summaries are fetched together (the loads do not depend on the running state), then
     // the state walks through them.
+    constexpr int kBatch = 8;
     const int end = first + nck;
-    for (int c0 = first; c0 < end; c0 += 4) {
-        float4 sa[4], sb[4];
-        float decay[4];
+    for (int c0 = first; c0 < end; c0 += kBatch) {
+        float4 sa[kBatch], sb[kBatch];
+        float decay[kBatch];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kBatch; ++i) {
             if (c0 + i < end) {
                 const size_t ch_head = (size_t)(c0 + i) * H + head;
                 const float4* sp = reinterpret_cast<const float4*>(p.ws_S + (ch_head * P + ch) * N + g * 8);
@@ -330,7 +351,7 @@ __global__ void __launch_bounds__(256) ssd_state_passing_kernel(const SsdPrefill
             }
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kBatch; ++i) {
             if (c0 + i < end) {
                 const size_t ch_head = (size_t)(c0 + i) * H + head;
                 // bf16 value and bf16 remainder of the incoming state: two operands, so that the product with C sees ~16 mantissa bits
@@ -361,58 +382,64 @@ __global__ void __launch_bounds__(256) ssd_state_passing_kernel(const SsdPrefill
 }
 
 // ---------------------------------------------------------------- kernel 3: outputs of a chunk
+// Shared memory is three operand tiles that are re-used as the phases go by:
+//   region A: C rows (operand of G and of C H_in^T)  ->  Xd (fetched from the workspace once those products are done)
+//   region B: B rows (operand of G)                   ->  masked G (operand of Y)
+//   region H: incoming state, value + remainder        ->  the z box (fetched once C H_in^T is done)
+//   regions A + B                                       ->  y rows on their way from accumulator lanes to channel-contiguous stores
 struct ScanSmem {
-    __nv_bfloat16 Ct[N / 8][Q][8];                       // C rows: A operand of G and of C H_in^T (K-major)
-    union {
-        __nv_bfloat16 Bt[N / 8][Q][8];                   // B rows: B operand of G (K-major) ...
-        __nv_bfloat16 M[Q / 8][Q][8];                    // ... then the masked G: A operand of Y (K-major over the source token)
-    };
-    unsigned char xd[(P / 8) * kXdColBytes];             // Xd = Delta u: B operand of Y (MN-major)
-    __nv_bfloat16 hin[2][N / 8][P][8];                   // incoming state, bf16 value and bf16 remainder: B operands of C H_in^T (K-major)
-    __nv_bfloat16 xs_ext[(Q + 3) * P];                   // 3 rows before the chunk + the x box
-    __nv_bfloat16 zs[Q * P];                             // the z box
-    float ystage[Q][P + 1];                              // y rows on their way from accumulator lanes to channel-contiguous stores
-    RowScalars rs;
-    uint64_t bar_in, bar_z, bar_g, bar_y;
+    unsigned char regA[N / 8 * Q * 16];   // C rows [N/8][Q][8] bf16 (K-major operand)  ->  Xd [(P/8)][Q + 1 unit][8] (MN-major operand, from kernel 1)
+    unsigned char regB[N / 8 * Q * 16];   // B rows [N/8][Q][8] bf16 (K-major operand)  ->  masked G [Q/8][Q][8] (K-major over the source token)
+    unsigned char regH[2 * N * P * 2];    // incoming state [2][N/8][P][8] bf16 (value, remainder; K-major operands)  ->  z box [Q][P] bf16
+    float csl[Q];                         // running log2-decay of the chunk's rows (from kernel 1)
+    uint64_t bar_in, bar_late, bar_g, bar_y;
     uint32_t tmem_base;
 };
+static_assert(sizeof(float) * Q * (P + 1) <= 2 * (N / 8 * Q * 16), "the y staging rows must fit the two operand tiles they lie over");
+static_assert((P / 8) * kXdColBytes <= N / 8 * Q * 16 && Q * P * 2 <= 2 * N * P * 2, "re-used regions too small");
 
-__global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
+__global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
     extern __shared__ __align__(1024) unsigned char s_raw[];
-    ScanSmem& sm = *reinterpret_cast<ScanSmem*>(s_raw + ((1024u - (smem_u32(s_raw) & 1023u)) & 1023u));
+    ScanSmem& sm = *reinterpret_cast<ScanSmem*>(s_raw + ((128u - (smem_u32(s_raw) & 127u)) & 127u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads, D = p.L.d_inner;
+    const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads;
     const ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, Q, cidx);
     if (ci.seq < 0) return;
     const int islot = load_slot(p.init_slot, ci.seq), fslot = load_slot(p.final_slot, ci.seq);
     if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;
     const int rows = ci.t1 - ci.t0;
+    const size_t ch_head = (size_t)cidx * H + head;
+    __nv_bfloat16 (*Ct)[Q][8] = reinterpret_cast<__nv_bfloat16 (*)[Q][8]>(sm.regA);
+    __nv_bfloat16 (*Bt)[Q][8] = reinterpret_cast<__nv_bfloat16 (*)[Q][8]>(sm.regB);
+    __nv_bfloat16 (*Mt)[Q][8] = reinterpret_cast<__nv_bfloat16 (*)[Q][8]>(sm.regB);
+    unsigned char* xd = sm.regA;
+    constexpr uint32_t kXdBytes = (P / 8) * kXdColBytes;
+    __nv_bfloat16* hin = reinterpret_cast<__nv_bfloat16*>(sm.regH);
+    __nv_bfloat16* zs = reinterpret_cast<__nv_bfloat16*>(sm.regH);
+    float (*ystage)[P + 1] = reinterpret_cast<float (*)[P + 1]>(sm.regA);   // runs on into regB
 
     if (tid == 0) {
-        mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_z, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_y, 1);
+        mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_late, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_y, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        mbar_expect_tx(&sm.bar_in, Q * P * 2 + 2 * Q * N * 2 + 2 * N * P * 2);
-        tma_box(sm.xs_ext + 3 * P, &maps.x, head * P, ci.t0, &sm.bar_in);
+        mbar_expect_tx(&sm.bar_in, 2 * Q * N * 2 + 2 * N * P * 2 + Q * 4);
 #pragma unroll
         for (int c = 0; c < N / 8; ++c) {
-            tma_box(&sm.Ct[c][0][0], &maps.C, c * 8, ci.t0, &sm.bar_in);
-            tma_box(&sm.Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_in);
+            tma_box(&Ct[c][0][0], &maps.C, c * 8, ci.t0, &sm.bar_in);
+            tma_box(&Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_in);
         }
-        bulk_load(&sm.hin[0][0][0][0], p.ws_hin + ((size_t)cidx * H + head) * 2 * N * P, 2 * N * P * 2, &sm.bar_in);
-        mbar_expect_tx(&sm.bar_z, Q * P * 2);
-        tma_box(sm.zs, &maps.z, head * P, ci.t0, &sm.bar_z);
+        bulk_load(hin, p.ws_hin + ch_head * 2 * N * P, 2 * N * P * 2, &sm.bar_in);
+        bulk_load(sm.csl, p.ws_csl + ch_head * Q, Q * 4, &sm.bar_in);
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 256); tc_fence_before(); }
-    load_halo(sm.xs_ext, p, ci, head, islot);
-    row_scalars(sm.rs, p, head, ci.t0, rows);
+    __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
     const uint32_t tG = tmem, tYi = tmem + 128, tYx = tmem + 192;   // accumulator columns: G, Y inside the chunk, C H_in^T
 
-    bool ok = mbar_wait_bounded(&sm.bar_in, 0u);
+    const bool ok = mbar_wait_bounded(&sm.bar_in, 0u);
     if (ok && tid == 0) {
         tc_fence_after();
-        const uint32_t c0 = smem_u32(&sm.Ct[0][0][0]), b0 = smem_u32(&sm.Bt[0][0][0]), h0 = smem_u32(&sm.hin[0][0][0][0]);
+        const uint32_t c0 = smem_u32(sm.regA), b0 = smem_u32(sm.regB), h0 = smem_u32(hin);
         constexpr uint32_t idG = instr_desc(Q, false, false), idX = instr_desc(P, false, false);
 #pragma unroll
         for (int k = 0; k < N / 16; ++k)   // G[t][s] = sum_n C[t][n] B[s][n]
@@ -425,24 +452,20 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefi
         }
         mma_commit(&sm.bar_g);
     }
-    // conv + SiLU of the warp's 32 rows; u stays in registers for the epilogue, Delta u goes to the operand buffer
-    float ua[kRowsPerWarp], ub[kRowsPerWarp];
-    if (ok) {
-        conv_rows(sm.xs_ext, p.L, head, [&](int r, int i, float a, float b) {
-            ua[i] = a; ub[i] = b;
-            const float dl = r < rows ? sm.rs.delta[r] : 0.0f;
-            const uint32_t v = r < rows ? pack_bf(dl * a, dl * b) : 0u;
-            *reinterpret_cast<uint32_t*>(sm.xd + (uint32_t)(lane >> 2) * kXdColBytes + (uint32_t)r * 16u + (uint32_t)(lane & 3) * 4u) = v;
-        });
+    const bool g_ok = ok && mbar_wait_bounded(&sm.bar_g, 0u);
+    if (g_ok && tid == 0) {
+        // both products that read C and the incoming state are complete: their tiles take Xd and the z box
+        mbar_expect_tx(&sm.bar_late, kXdBytes + Q * P * 2);
+        bulk_load(xd, p.ws_xd + ch_head * (kXdBytes / 2), kXdBytes, &sm.bar_late);
+        tma_box(zs, &maps.z, head * P, ci.t0, &sm.bar_late);
     }
-    bool g_ok = ok && mbar_wait_bounded(&sm.bar_g, 0u);
     if (g_ok) {
         tc_fence_after();
-        // row t of G, masked: M[t][s] = G[t][s] exp(cs_t - cs_s) for s <= t, else 0; written over the B boxes (G is complete)
-        // warps w and w + 4 own rows 32 (w % 4) ..: the first takes column blocks 0 and 3, the second 1 and 2 (five
-        // non-zero blocks of 32 x 32 on each side of the split)
+        // row t of G, masked: M[t][s] = G[t][s] exp(cs_t - cs_s) for s <= t, else 0; written over the B boxes (G is complete).
+        // Warps w and w + 4 own rows 32 (w % 4) ..: the first takes column blocks 0 and 3, the second 1 and 2 (five
+        // non-zero blocks of 32 x 32 on each side of the split).
         const int rb = warp & 3, row = rb * 32 + lane;
-        const float my = sm.rs.csl[row];
+        const float my = sm.csl[row];
 #pragma unroll 1
         for (int q = 0; q < 2; ++q) {
             const int cb = warp < 4 ? (q == 0 ? 0 : 3) : (q == 0 ? 1 : 2);
@@ -453,8 +476,8 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefi
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
                     const int s0 = cb * 32 + j;
-                    const float m0 = s0 <= row ? g[j] * ex2(my - sm.rs.csl[s0]) : 0.0f;
-                    const float m1 = s0 + 1 <= row ? g[j + 1] * ex2(my - sm.rs.csl[s0 + 1]) : 0.0f;
+                    const float m0 = s0 <= row ? g[j] * ex2(my - sm.csl[s0]) : 0.0f;
+                    const float m1 = s0 + 1 <= row ? g[j + 1] * ex2(my - sm.csl[s0 + 1]) : 0.0f;
                     packed[j >> 1] = pack_bf(m0, m1);
                 }
             } else {
@@ -463,58 +486,64 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_scan_kernel(const SsdPrefi
             }
 #pragma unroll
             for (int u4 = 0; u4 < 4; ++u4)
-                *reinterpret_cast<uint4*>(&sm.M[cb * 4 + u4][row][0]) = make_uint4(packed[4 * u4], packed[4 * u4 + 1], packed[4 * u4 + 2], packed[4 * u4 + 3]);
+                *reinterpret_cast<uint4*>(&Mt[cb * 4 + u4][row][0]) = make_uint4(packed[4 * u4], packed[4 * u4 + 1], packed[4 * u4 + 2], packed[4 * u4 + 3]);
         }
     }
+    const bool late_ok = g_ok && mbar_wait_bounded(&sm.bar_late, 0u);
     fence_async_smem();
     tc_fence_before();
-    const bool all_ok = !__syncthreads_or(!g_ok);
+    const bool all_ok = !__syncthreads_or(!late_ok);
     if (all_ok && tid == 0) {
         tc_fence_after();
-        const uint32_t m0 = smem_u32(&sm.M[0][0][0]), x0 = smem_u32(sm.xd);
+        const uint32_t m0 = smem_u32(sm.regB), x0 = smem_u32(xd);
         constexpr uint32_t idY = instr_desc(P, false, true);
 #pragma unroll
         for (int k = 0; k < Q / 16; ++k)   // Yi[t][p] = sum_s M[t][s] Xd[s][p]
             mma_bf16(tYi, operand_desc(m0 + k * 2 * kColBytes, kColBytes, 128), operand_desc(x0 + k * 256, 128, kXdColBytes), idY, k > 0);
         mma_commit(&sm.bar_y);
     }
+    // skip term inputs of the warp's rows travel while the product runs: u of this lane's channel pair (from kernel 1)
+    const int d = head * P + 2 * lane;
+    uint32_t uraw[kRowsPerWarp];
+#pragma unroll
+    for (int i = 0; i < kRowsPerWarp; ++i) {
+        const int r = warp * kRowsPerWarp + i;
+        uraw[i] = (all_ok && r < rows) ? *reinterpret_cast<const uint32_t*>(p.ws_u + (size_t)(ci.t0 + r) * p.L.d_inner + d) : 0u;
+    }
     bool y_ok = all_ok && mbar_wait_bounded(&sm.bar_y, 0u);
     if (y_ok) {
         tc_fence_after();
         const int rb = warp & 3, row = rb * 32 + lane, half = warp >> 2;
-        const float scale = ex2(sm.rs.csl[row]);   // decay from the chunk's start through this row
+        const float scale = ex2(sm.csl[row]);   // decay from the chunk's start through this row
         float yi[32], yx[32];
         tmem_ld32(tYi + ((uint32_t)(rb * 32) << 16) + half * 32, yi);
         tmem_ld32(tYx + ((uint32_t)(rb * 32) << 16) + half * 32, yx);
+        __syncwarp();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) sm.ystage[row][half * 32 + j] = fmaf(scale, yx[j], yi[j]);
+        for (int j = 0; j < 32; ++j) yi[j] = fmaf(scale, yx[j], yi[j]);
+        // the staging rows lie over the operand tiles of the product that has just completed
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ystage[row][half * 32 + j] = yi[j];
     }
     y_ok = !__syncthreads_or(!y_ok);
-    const bool z_ok = y_ok && mbar_wait_bounded(&sm.bar_z, 0u);
-    if (z_ok) {
+    if (y_ok) {
         // skip term, gate, store: the warp's rows, this lane's channel pair (128 contiguous bytes per row and warp)
-        const int d = head * P + 2 * lane;
         const float da = p.L.D ? __ldg(p.L.D + d) : 0.0f, db = p.L.D ? __ldg(p.L.D + d + 1) : 0.0f;
-        const uint32_t* zc = reinterpret_cast<const uint32_t*>(sm.zs) + lane;
+        const uint32_t* zc = reinterpret_cast<const uint32_t*>(zs) + lane;
 #pragma unroll
         for (int i = 0; i < kRowsPerWarp; ++i) {
             const int r = warp * kRowsPerWarp + i;
             if (r < rows) {
                 const uint32_t zv = zc[r * (P / 2)];
-                const float oa = fmaf(da, ua[i], sm.ystage[r][2 * lane]) * silu(bf_lo(zv));
-                const float ob = fmaf(db, ub[i], sm.ystage[r][2 * lane + 1]) * silu(bf_hi(zv));
+                const float oa = fmaf(da, bf_lo(uraw[i]), ystage[r][2 * lane]) * silu(bf_lo(zv));
+                const float ob = fmaf(db, bf_hi(uraw[i]), ystage[r][2 * lane + 1]) * silu(bf_hi(zv));
                 *reinterpret_cast<uint32_t*>(p.out + (size_t)(ci.t0 + r) * p.ldo + d) = pack_bf(oa, ob);
             }
         }
-        // the sequence's last chunk leaves the window: the last three raw inputs (extended rows rows .. rows + 2)
-        if (ci.k == ci.nck - 1 && fslot >= 0 && warp < 3) {
-            __nv_bfloat16* dc = static_cast<__nv_bfloat16*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride + (size_t)warp * D + d;
-            *reinterpret_cast<uint32_t*>(dc) = reinterpret_cast<const uint32_t*>(sm.xs_ext)[(rows + warp) * (P / 2) + lane];
-        }
     } else if (tid == 0) {
         flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
-        if (!ok) mbar_wait_bounded(&sm.bar_in, 0u);
-        mbar_wait_bounded(&sm.bar_z, 0u);
+        if (!ok) mbar_wait_bounded(&sm.bar_in, 0u);   // copies target this block's shared memory: one more bounded chance
+        if (g_ok && !late_ok) mbar_wait_bounded(&sm.bar_late, 0u);
     }
     tc_fence_before();
     __syncthreads();
@@ -531,13 +560,13 @@ cudaError_t allow_smem(K kernel, size_t bytes) {
 cudaError_t launch_ssd_prefill(const SsdPrefillArgs& p, const SsdMaps& maps, cudaStream_t st) {
     const int H = p.L.n_heads;
     cudaError_t e;
-    constexpr size_t smem1 = sizeof(StateSmem) + 1024, smem3 = sizeof(ScanSmem) + 1024;
+    constexpr size_t smem1 = sizeof(StateSmem) + 1024, smem3 = sizeof(ScanSmem) + 128;
     if ((e = allow_smem(ssd_chunk_state_kernel, smem1)) != cudaSuccess) return e;
     if ((e = allow_smem(ssd_chunk_scan_kernel, smem3)) != cudaSuccess) return e;
     dim3 grid(H, p.n_chunks_bound);
     ssd_chunk_state_kernel<<<grid, kThreads, smem1, st>>>(p, maps);
-    dim3 g2((p.L.d_inner * (N / 8) + 255) / 256, p.n_seq);
-    ssd_state_passing_kernel<<<g2, 256, 0, st>>>(p);
+    dim3 g2((p.L.d_inner * (N / 8) + 127) / 128, p.n_seq);
+    ssd_state_passing_kernel<<<g2, 128, 0, st>>>(p);
     ssd_chunk_scan_kernel<<<grid, kThreads, smem3, st>>>(p, maps);
     return cudaGetLastError();
 }
