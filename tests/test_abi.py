@@ -172,3 +172,58 @@ def test_prefill_plan_seen_through_the_workspace_query(lib):
     o = binding._PrefillOpts(chunk_len=64, block_channels=0)
     assert q(2048, 1, 2048, C.byref(o)) >= 32 * per_chunk      # a forced chunk length is honoured
     assert q(0, 1, 8) == 0 and q(8, 0, 8) == 0     # nonsense sizes give 0, not garbage
+
+
+def test_ssd_host_side_checks(lib):
+    """The SSD entry points turn unsupported shapes and bad arguments away before any launch."""
+    from paper_2506_01206_b200 import binding
+    INVALID, UNSUPPORTED, MISALIGNED, WORKSPACE = -1, -2, -3, -4
+
+    def layer(**kw):
+        base = dict(d_inner=128, headdim=64, d_state=128, d_conv=4, act=1, flags=1, A=0x1000, D=0, conv_w=0x2000, conv_b=0, dt_bias=0)
+        base.update(kw)
+        return binding._SsdLayer(*[base[k] for k in ("d_inner", "headdim", "d_state", "d_conv", "act", "flags", "A", "D", "conv_w", "conv_b", "dt_bias")])
+
+    cache = _cache(binding, ssm_slot_stride=128 * 128, ssm_layer_stride=4 * 128 * 128, conv_slot_stride=3 * 128, conv_layer_stride=12 * 128)
+
+    def prefill(lay=None, cache=cache, T=300, n_seq=1, x=0x100000, ldx=128, dt=0x300000, lddt=2, B=0x400000, ldb=128, ws=0x900000, ws_bytes=1 << 30, cu=None):
+        lay = lay or layer()
+        return lib.mdraft_ssd_prefill(C.byref(lay), C.byref(cache) if cache is not None else None, 0, x, ldx, 0x200000, 128, dt, lddt, B, ldb,
+                                      0x500000, 128, 0x600000, 128, T, n_seq, cu, None, 0x800000, ws, ws_bytes, None, None)
+
+    ok = layer()
+    need = lib.mdraft_ssd_prefill_workspace_bytes(C.byref(ok), 300, 1)
+    assert need > 0 and need % 256 == 0
+    assert lib.mdraft_ssd_prefill_workspace_bytes(C.byref(layer(headdim=32)), 300, 1) == 0
+    assert prefill(lay=layer(headdim=32)) == UNSUPPORTED
+    assert prefill(lay=layer(d_state=16)) == UNSUPPORTED
+    assert prefill(lay=layer(act=0)) == UNSUPPORTED            # bf16 activations only
+    assert prefill(lay=layer(d_inner=96)) == UNSUPPORTED       # whole heads only
+    assert prefill(lay=layer(flags=2)) == INVALID              # only the softplus flag has a meaning here
+    assert prefill(lay=layer(A=0)) == INVALID
+    assert prefill(x=None) == INVALID
+    assert prefill(lddt=1) == INVALID                          # dt rows shorter than the head count
+    assert prefill(ldb=64) == INVALID
+    assert prefill(B=0x400008) == MISALIGNED
+    assert prefill(ws=None) == WORKSPACE
+    assert prefill(ws_bytes=need - 1) == WORKSPACE
+    assert prefill(ws=0x900010) == MISALIGNED
+    assert prefill(n_seq=2) == INVALID                         # offsets may be left out for one sequence only
+    small = _cache(binding)                                    # slots sized for 16 states
+    assert prefill(cache=small) == INVALID
+    assert prefill(n_seq=0, T=0) == 0
+
+    def step(lay=None, cache=cache, n=2, par=0x700000, nod=0x800000, n_levels=1, levels=None, lddt=2):
+        lay = lay or layer()
+        return lib.mdraft_ssd_tree_step(C.byref(lay), C.byref(cache) if cache is not None else None, 0, 0x100000, 128, 0x200000, 128, 0x300000, lddt,
+                                        0x400000, 128, 0x500000, 128, 0x600000, 128, n, par, nod, n_levels, levels, None, None)
+
+    assert step(cache=None) == INVALID
+    assert step(par=None) == INVALID
+    assert step(n=0) == 0
+    assert step(n_levels=2) == INVALID
+    assert step(lay=layer(d_conv=3)) == UNSUPPORTED
+    assert step(lddt=1) == INVALID
+    # the commit call moves 128-state slots too, and nothing between the two sizes
+    commit = lambda ds: lib.mdraft_state_commit(C.byref(cache), 128, ds, 4, 1, 0, None, None, None, None)
+    assert commit(128) == 0 and commit(64) == UNSUPPORTED
