@@ -195,3 +195,62 @@ def test_ssd_bad_slots_are_flagged_not_followed():
     md.mdraft_ssd_tree_step(lay, cache, 0, *[t[:1] for t in dev], out[:1], i32([5]), i32([0]), None, status)
     torch.cuda.synchronize()
     assert int(status.item()) & md.MDRAFT_DEV_BAD_SLOT
+
+
+def _ssd_case(seed):
+    g = np.random.default_rng(5000 + seed)
+    Dn = int(g.choice([64, 128, 192, 320]))
+    S = int(g.integers(1, 5))
+    lens = [int(v) for v in g.choice([0, 1, 2, 3, 5, 31, 64, 127, 128, 129, 200, 257, 300], size=S)]
+    if sum(lens) == 0:
+        lens[0] = 17
+    return dict(Dn=Dn, lens=lens, conv_bias=bool(g.random() < 0.5), softplus=bool(g.random() < 0.75),
+                init=str(g.choice(["none", "slots", "mixed"])), regime=str(g.choice(["recipe", "recipe", "big_dt", "A_zero", "A_steep"])), seed=seed)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_ssd_prefill_case(seed):
+    """Seeded sweep over widths, packed length mixes around the chunk size, starting-slot arrangements and value regimes
+    outside the recipe (pre-activations from -60 to +30 under softplus; heads with A = 0; A down to -200)."""
+    c = _ssd_case(seed)
+    cfg, prm, arrs, cu = make(c["Dn"], c["lens"], seed=seed, conv_bias=c["conv_bias"])
+    x, z, dt, B, C = arrs
+    S, Dn = len(c["lens"]), c["Dn"]
+    g = np.random.default_rng(6000 + seed)
+    H = Dn // P
+    flags = md.MDRAFT_DT_SOFTPLUS if c["softplus"] else 0
+    if c["regime"] == "A_zero":
+        prm.A[::2] = 0.0
+    elif c["regime"] == "A_steep":
+        prm.A[:] = -g.uniform(40.0, 200.0, size=H).astype(np.float32)
+    if not c["softplus"]:
+        dt = gen.round_to_act(np.where(g.random(dt.shape) < 0.3, 0.0, np.abs(dt) * 0.05).astype(np.float32), "bf16")
+        prm.dt_bias[:] = 0
+    elif c["regime"] == "big_dt":
+        kind = g.integers(0, 3, size=dt.shape)
+        dt = gen.round_to_act(np.where(kind == 0, dt, np.where(kind == 1, g.uniform(10.0, 30.0, size=dt.shape), g.uniform(-60.0, -10.0, size=dt.shape))).astype(np.float32), "bf16")
+        prm.dt_bias[:] = 0
+    arrs = (x, z, dt, B, C)
+    h0 = g.normal(size=(S, Dn, N)).astype(np.float32)
+    c0 = gen.round_to_act(g.normal(size=(S, 3, Dn)).astype(np.float32), "bf16")
+    init = None if c["init"] == "none" else (np.arange(S) if c["init"] == "slots" else np.where(g.random(S) < 0.5, np.arange(S), -1))
+    lay = upload_ssd_layer(prm, flags)
+    cache = ssd_cache(2 * S, Dn)
+    cache.ssm.fill_(float("nan")); cache.conv.fill_(float("nan"))
+    cache.ssm[0, :S] = torch.from_numpy(h0).cuda(); cache.conv[0, :S] = to_device(c0, BF)
+    T = int(cu[-1])
+    out = torch.full((T, Dn), float("nan"), dtype=BF, device="cuda")
+    ws = torch.empty(max(256, md.mdraft_ssd_prefill_workspace_bytes(lay, T, S)), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    md.mdraft_ssd_prefill(lay, cache, 0, *[to_device(a, BF) for a in arrs], out, i32(cu), None if init is None else i32(init), i32(np.arange(S, 2 * S)), ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o_ci = np.zeros((S, 3, Dn)); o_hi = np.zeros((S, Dn, N))
+    if init is not None:
+        for s_ in range(S):
+            if init[s_] >= 0:
+                o_ci[s_] = c0[s_]; o_hi[s_] = h0[s_]
+    o_out, o_conv, o_h = oracle.ssd_prefill(oracle.ssd_layer_from_params(prm, flags=flags & 1), *arrs, cu_seqlens=cu, conv_init=o_ci, h_init=o_hi)
+    assert_close(out.float().cpu().numpy(), o_out, TOL["bf16"], f"out ({c})")
+    assert_close(cache.ssm[0, S:].cpu().numpy(), o_h, TOL_STATE, f"state ({c})")
+    assert np.array_equal(cache.conv[0, S:].float().cpu().numpy().astype(np.float64), o_conv), f"window ({c})"
