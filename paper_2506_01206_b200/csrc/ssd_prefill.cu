@@ -117,6 +117,12 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Programmatic dependent launch: the kernels of a call (and the first kernel of the next call on the stream) may start
+// before the kernel ahead of them has finished.  A kernel passes grid_wait() before it touches anything a kernel ahead
+// of it writes, or overwrites anything one reads; every block passes it on every path, so that a kernel's completion
+// implies the completion of everything before it.
+__device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
@@ -177,25 +183,31 @@ __device__ __forceinline__ void load_halo(__nv_bfloat16* xs_ext, const SsdPrefil
     *reinterpret_cast<uint32_t*>(xs_ext + j * P + 2 * lane) = v;
 }
 
-// conv + SiLU of the warp's kRowsPerWarp rows for this lane's channel pair; calls f(row, index in the warp, u_lo, u_hi).
+// The warp's rows of the extended x tile (its kRowsPerWarp rows and the three before them) for this lane's channel pair.
+__device__ __forceinline__ void load_rows(const __nv_bfloat16* xs_ext, uint32_t (&xr)[kRowsPerWarp + 3]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t* col = reinterpret_cast<const uint32_t*>(xs_ext) + lane;   // row r of the chunk is extended row r + 3
+    const int r0 = warp * kRowsPerWarp;
+#pragma unroll
+    for (int i = 0; i < kRowsPerWarp + 3; ++i) xr[i] = col[(r0 + i) * (P / 2)];
+}
+
+// conv + SiLU of those rows; calls f(row, index in the warp, u_lo, u_hi).
 template <typename F>
-__device__ __forceinline__ void conv_rows(const __nv_bfloat16* xs_ext, const SsdLayerDev& L, int head, F&& f) {
+__device__ __forceinline__ void conv_rows(const uint32_t (&xr)[kRowsPerWarp + 3], const SsdLayerDev& L, int head, F&& f) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int d = head * P + 2 * lane;
     const float4 wa = __ldg(reinterpret_cast<const float4*>(L.conv_w + (size_t)d * kW));
     const float4 wb = __ldg(reinterpret_cast<const float4*>(L.conv_w + (size_t)(d + 1) * kW));
     const float ba = L.conv_b ? __ldg(L.conv_b + d) : 0.0f, bb = L.conv_b ? __ldg(L.conv_b + d + 1) : 0.0f;
-    const uint32_t* col = reinterpret_cast<const uint32_t*>(xs_ext) + lane;   // row r of the chunk is extended row r + 3
     const int r0 = warp * kRowsPerWarp;
-    uint32_t w0 = col[(r0 + 0) * (P / 2)], w1 = col[(r0 + 1) * (P / 2)], w2 = col[(r0 + 2) * (P / 2)];
 #pragma unroll
     for (int i = 0; i < kRowsPerWarp; ++i) {
-        const uint32_t xv = col[(r0 + i + 3) * (P / 2)];
+        const uint32_t w0 = xr[i], w1 = xr[i + 1], w2 = xr[i + 2], xv = xr[i + 3];
         float a = fmaf(wa.x, bf_lo(w0), ba), b = fmaf(wb.x, bf_hi(w0), bb);
         a = fmaf(wa.y, bf_lo(w1), a); b = fmaf(wb.y, bf_hi(w1), b);
         a = fmaf(wa.z, bf_lo(w2), a); b = fmaf(wb.z, bf_hi(w2), b);
         a = fmaf(wa.w, bf_lo(xv), a); b = fmaf(wb.w, bf_hi(xv), b);
-        w0 = w1; w1 = w2; w2 = xv;
         f(r0 + i, i, silu(a), silu(b));
     }
 }
@@ -204,73 +216,85 @@ __device__ __forceinline__ void conv_rows(const __nv_bfloat16* xs_ext, const Ssd
 struct StateSmem {
     __nv_bfloat16 Bt[N / 8][Q][8];                        // B rows of the chunk, one TMA box per 8 states
     unsigned char xw_hi[(P / 8) * kXdColBytes];           // Xw = Delta exp(cs_end - cs) u, bf16 value ...
-    unsigned char xw_lo[(P / 8) * kXdColBytes];           // ... and bf16 remainder
-    unsigned char xd[(P / 8) * kXdColBytes];              // Xd = Delta u, the operand of the chunk-scan kernel (sent to the workspace)
-    __nv_bfloat16 xs_ext[(Q + 3) * P];                    // 3 rows before the chunk + the x box
+    // ... and bf16 remainder, which takes the place of the x tile (3 rows before the chunk + the x box) once every thread
+    // holds its rows of x in registers
+    unsigned char xs_or_lo[(Q + 3) * P * 2];
     RowScalars rs;
     uint64_t bar_tma, bar_mma;
     uint32_t tmem_base;
 };
+static_assert((Q + 3) * P * 2 >= (P / 8) * kXdColBytes, "the remainder operand must fit the x tile it replaces");
+static_assert(3 * (sizeof(StateSmem) + 128 + 1024) <= 227 * 1024, "three blocks per SM");
 
-__global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
+__global__ void __launch_bounds__(kThreads, 3) ssd_chunk_state_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
     extern __shared__ __align__(1024) unsigned char s_raw[];
-    StateSmem& sm = *reinterpret_cast<StateSmem*>(s_raw + ((1024u - (smem_u32(s_raw) & 1023u)) & 1023u));
+    StateSmem& sm = *reinterpret_cast<StateSmem*>(s_raw + ((128u - (smem_u32(s_raw) & 127u)) & 127u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads;
+    // The inputs may be the work of the kernel ahead of this call, and the workspace is still being read by the call
+    // before this one: nothing is touched before that kernel is complete.  Only then may the next kernels start, which
+    // lets them read the call's inputs without a wait of their own.
+    grid_wait();
+    grid_release_dependents();
     const ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, Q, cidx);
     if (ci.seq < 0) return;
     const int islot = load_slot(p.init_slot, ci.seq), fslot = load_slot(p.final_slot, ci.seq);
     if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;   // reported by the state-passing kernel
     const int rows = ci.t1 - ci.t0;
+    __nv_bfloat16* xs_ext = reinterpret_cast<__nv_bfloat16*>(sm.xs_or_lo);
+    unsigned char* xw_lo = sm.xs_or_lo;
 
     if (tid == 0) {
         mbar_init(&sm.bar_tma, 1);
         mbar_init(&sm.bar_mma, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         mbar_expect_tx(&sm.bar_tma, Q * P * 2 + Q * N * 2);
-        tma_box(sm.xs_ext + 3 * P, &maps.x, head * P, ci.t0, &sm.bar_tma);
+        tma_box(xs_ext + 3 * P, &maps.x, head * P, ci.t0, &sm.bar_tma);
 #pragma unroll
         for (int c = 0; c < N / 8; ++c) tma_box(&sm.Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_tma);
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 64); tc_fence_before(); }
-    load_halo(sm.xs_ext, p, ci, head, islot);
+    load_halo(xs_ext, p, ci, head, islot);
     row_scalars(sm.rs, p, head, ci.t0, rows);   // two block-wide barriers inside: barrier init and tmem_base are visible after it
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
     bool ok = mbar_wait_bounded(&sm.bar_tma, 0u);
+    uint32_t xr[kRowsPerWarp + 3];
+    if (ok) {
+        load_rows(xs_ext, xr);
+        // the sequence's last chunk leaves the window: the last three raw inputs (extended rows rows .. rows + 2)
+        if (ci.k == ci.nck - 1 && fslot >= 0 && warp < 3) {
+            __nv_bfloat16* dc = static_cast<__nv_bfloat16*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride + (size_t)warp * p.L.d_inner + head * P + 2 * lane;
+            *reinterpret_cast<uint32_t*>(dc) = reinterpret_cast<const uint32_t*>(xs_ext)[(rows + warp) * (P / 2) + lane];
+        }
+    }
+    __syncthreads();   // every thread holds its rows: the x tile may be overwritten
     if (ok) {
         const float cs_end_l = sm.rs.csl[Q - 1];
-        conv_rows(sm.xs_ext, p.L, head, [&](int r, int, float ua, float ub) {
+        unsigned char* xd_g = reinterpret_cast<unsigned char*>(p.ws_xd) + ((size_t)cidx * H + head) * ((P / 8) * kXdColBytes);
+        conv_rows(xr, p.L, head, [&](int r, int, float ua, float ub) {
             const float wgt = r < rows ? sm.rs.delta[r] * ex2(cs_end_l - sm.rs.csl[r]) : 0.0f;
             const float va = r < rows ? wgt * ua : 0.0f, vb = r < rows ? wgt * ub : 0.0f;
             const uint32_t hi = pack_bf(va, vb);
             const uint32_t lo = pack_bf(va - bf_lo(hi), vb - bf_hi(hi));
             const uint32_t off = (uint32_t)(lane >> 2) * kXdColBytes + (uint32_t)r * 16u + (uint32_t)(lane & 3) * 4u;
             *reinterpret_cast<uint32_t*>(sm.xw_hi + off) = hi;
-            *reinterpret_cast<uint32_t*>(sm.xw_lo + off) = lo;
+            *reinterpret_cast<uint32_t*>(xw_lo + off) = lo;
+            // Xd = Delta u goes straight to the workspace, in the layout of the chunk-scan kernel's operand
             const float dl = r < rows ? sm.rs.delta[r] : 0.0f;
-            *reinterpret_cast<uint32_t*>(sm.xd + off) = r < rows ? pack_bf(dl * ua, dl * ub) : 0u;
+            *reinterpret_cast<uint32_t*>(xd_g + off) = r < rows ? pack_bf(dl * ua, dl * ub) : 0u;
             if (r < rows) *reinterpret_cast<uint32_t*>(p.ws_u + (size_t)(ci.t0 + r) * p.L.d_inner + head * P + 2 * lane) = pack_bf(ua, ub);
         });
         if (tid < Q) p.ws_csl[((size_t)cidx * H + head) * Q + tid] = sm.rs.csl[tid];
-        // the sequence's last chunk leaves the window: the last three raw inputs (extended rows rows .. rows + 2)
-        if (ci.k == ci.nck - 1 && fslot >= 0 && warp < 3) {
-            __nv_bfloat16* dc = static_cast<__nv_bfloat16*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride + (size_t)warp * p.L.d_inner + head * P + 2 * lane;
-            *reinterpret_cast<uint32_t*>(dc) = reinterpret_cast<const uint32_t*>(sm.xs_ext)[(rows + warp) * (P / 2) + lane];
-        }
     }
-    fence_async_smem();   // the operands written by threads must be visible to the tensor core's and the copy engine's reads
+    fence_async_smem();   // the operands written by threads must be visible to the tensor core's reads
     const bool all_ok = !__syncthreads_or(!ok);
     if (all_ok && tid == 0) {
-        // Xd leaves for the workspace as one bulk store (same bytes, same layout as the chunk-scan kernel's operand)
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(p.ws_xd + ((size_t)cidx * H + head) * (sizeof(sm.xd) / 2))),
-                     "r"(smem_u32(sm.xd)), "r"((uint32_t)sizeof(sm.xd)) : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         tc_fence_after();
         // S^T (n x p) = sum over tokens: A operand = B^T read MN-major out of the TMA boxes, B operand = Xw MN-major.
         constexpr uint32_t idesc = instr_desc(P, true, true);
-        const uint32_t a0 = smem_u32(&sm.Bt[0][0][0]), bh = smem_u32(sm.xw_hi), bl = smem_u32(sm.xw_lo);
+        const uint32_t a0 = smem_u32(&sm.Bt[0][0][0]), bh = smem_u32(sm.xw_hi), bl = smem_u32(xw_lo);
 #pragma unroll
         for (int k = 0; k < Q / 16; ++k)
             mma_bf16(tmem, operand_desc(a0 + k * 256, 128, kColBytes), operand_desc(bh + k * 256, 128, kXdColBytes), idesc, k > 0);
@@ -297,19 +321,25 @@ __global__ void __launch_bounds__(kThreads) ssd_chunk_state_kernel(const SsdPref
         flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
         if (!ok) mbar_wait_bounded(&sm.bar_tma, 0u);   // the copies target this block's shared memory: one more bounded chance
     }
-    if (all_ok && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory stays valid until the store has read it
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_free(tmem, 64);
 }
 
 // ---------------------------------------------------------------- kernel 2: chain the chunk states of a sequence
-// Thread = (channel d, group of 8 states).  Walks the sequence's chunks in order: writes the chunk's incoming state as
-// bf16 (a value and a remainder) in the operand layout [state group][channel of the head][8], then h <- exp(chunk decay) h + S.
-__global__ void __launch_bounds__(128) ssd_state_passing_kernel(const SsdPrefillArgs p) {
+// Thread = (channel d, 4 states); a lane pair covers one 16-byte unit of the operand.  Walks the sequence's chunks in order:
+// writes the chunk's incoming state as bf16 (a value and a remainder) in the operand layout [state group][channel of the
+// head][8], then h <- exp(chunk decay) h + S.
+constexpr int kPassThreads = 128;
+constexpr int kPassBatch = 16;   // chunks whose summaries are in flight together
+
+__global__ void __launch_bounds__(kPassThreads) ssd_state_passing_kernel(const SsdPrefillArgs p) {
     const int D = p.L.d_inner, H = p.L.n_heads;
     const int s = blockIdx.y;
-    const int idx = blockIdx.x * 128 + threadIdx.x;
+    const int idx = blockIdx.x * kPassThreads + threadIdx.x;
+    grid_release_dependents();
+    // Sequence offsets, slots and the starting state are inputs of the call: the kernel ahead let this one start only
+    // after everything before the call had finished, so they are read before the wait below.
     int first, nck;
     seq_chunks(p.cu, p.n_seq, p.T, Q, s, first, nck);   // whole warps call this
     // malformed offsets: the sequence has no chunk and is skipped
@@ -318,63 +348,48 @@ __global__ void __launch_bounds__(128) ssd_state_passing_kernel(const SsdPrefill
         if (lo < 0 || hi < lo || hi > p.T) flag(p.dev_status, MDRAFT_DEV_BAD_SEQLENS);
     }
     const int islot = load_slot(p.init_slot, s), fslot = load_slot(p.final_slot, s);
-    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
-        return;
-    }
-    if (idx >= D * (N / 8)) return;
-    // consecutive threads: consecutive channels of one head and one state group, so that the 16-byte operand words they
-    // write are contiguous (their 32-byte reads of the chunk states each fill a sector of their own)
-    const int ch = idx % P, g = (idx / P) % (N / 8), head = idx / (P * (N / 8)), d = head * P + ch;
-    float h[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) h[i] = 0.0f;
-    if (islot >= 0) {
-        const float4* src = reinterpret_cast<const float4*>(p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)d * N + g * 8);
-        const float4 a = src[0], b = src[1];
-        h[0] = a.x; h[1] = a.y; h[2] = a.z; h[3] = a.w; h[4] = b.x; h[5] = b.y; h[6] = b.z; h[7] = b.w;
-    }
-    // Eight chunks per round: their summaries are fetched together (the loads do not depend on the running state), then
-    // the state walks through them.
-    constexpr int kBatch = 8;
+    const bool slots_ok = islot < p.pool.n_slots && fslot < p.pool.n_slots;
+    if (!slots_ok && blockIdx.x == 0 && threadIdx.x == 0) flag(p.dev_status, MDRAFT_DEV_BAD_SLOT);
+    const bool mine = slots_ok && idx < D * (N / 4);
+    // consecutive lanes: the two halves of a unit, then consecutive channels of one head and one state group, so that the
+    // 16-byte operand units a warp writes are contiguous (its 32-byte reads of the chunk states each fill a sector)
+    const int sub = idx & 1, ch = (idx >> 1) % P, g = (idx / (2 * P)) % (N / 8), head = mine ? idx / (2 * P * (N / 8)) : 0, d = head * P + ch;
+    const int n0 = g * 8 + sub * 4;
+    float4 h = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    if (mine && islot >= 0) h = *reinterpret_cast<const float4*>(p.pool.ssm + (size_t)islot * p.pool.ssm_slot_stride + (size_t)d * N + n0);
+    grid_wait();   // the chunk states are the work of the kernel just before
+    if (!mine) return;
     const int end = first + nck;
-    for (int c0 = first; c0 < end; c0 += kBatch) {
-        float4 sa[kBatch], sb[kBatch];
-        float decay[kBatch];
+    for (int c0 = first; c0 < end; c0 += kPassBatch) {
+        float4 sv[kPassBatch];
+        float decay[kPassBatch];
 #pragma unroll
-        for (int i = 0; i < kBatch; ++i) {
+        for (int i = 0; i < kPassBatch; ++i) {
             if (c0 + i < end) {
                 const size_t ch_head = (size_t)(c0 + i) * H + head;
-                const float4* sp = reinterpret_cast<const float4*>(p.ws_S + (ch_head * P + ch) * N + g * 8);
-                sa[i] = sp[0]; sb[i] = sp[1];
+                sv[i] = *reinterpret_cast<const float4*>(p.ws_S + (ch_head * P + ch) * N + n0);
                 decay[i] = __ldg(p.ws_decay + ch_head);
             }
         }
 #pragma unroll
-        for (int i = 0; i < kBatch; ++i) {
+        for (int i = 0; i < kPassBatch; ++i) {
             if (c0 + i < end) {
                 const size_t ch_head = (size_t)(c0 + i) * H + head;
                 // bf16 value and bf16 remainder of the incoming state: two operands, so that the product with C sees ~16 mantissa bits
-                uint4 hi4, lo4;
-                hi4.x = pack_bf(h[0], h[1]); hi4.y = pack_bf(h[2], h[3]); hi4.z = pack_bf(h[4], h[5]); hi4.w = pack_bf(h[6], h[7]);
-                lo4.x = pack_bf(h[0] - bf_lo(hi4.x), h[1] - bf_hi(hi4.x)); lo4.y = pack_bf(h[2] - bf_lo(hi4.y), h[3] - bf_hi(hi4.y));
-                lo4.z = pack_bf(h[4] - bf_lo(hi4.z), h[5] - bf_hi(hi4.z)); lo4.w = pack_bf(h[6] - bf_lo(hi4.w), h[7] - bf_hi(hi4.w));
-                __nv_bfloat16* blob = p.ws_hin + ch_head * 2 * N * P;
-                *reinterpret_cast<uint4*>(blob + ((size_t)g * P + ch) * 8) = hi4;
-                *reinterpret_cast<uint4*>(blob + (size_t)N * P + ((size_t)g * P + ch) * 8) = lo4;
+                uint2 hi2, lo2;
+                hi2.x = pack_bf(h.x, h.y); hi2.y = pack_bf(h.z, h.w);
+                lo2.x = pack_bf(h.x - bf_lo(hi2.x), h.y - bf_hi(hi2.x)); lo2.y = pack_bf(h.z - bf_lo(hi2.y), h.w - bf_hi(hi2.y));
+                __nv_bfloat16* blob = p.ws_hin + ch_head * 2 * N * P + ((size_t)g * P + ch) * 8 + sub * 4;
+                *reinterpret_cast<uint2*>(blob) = hi2;
+                *reinterpret_cast<uint2*>(blob + (size_t)N * P) = lo2;
                 const float dk = ex2(decay[i] * kLog2e);
-                h[0] = fmaf(dk, h[0], sa[i].x); h[1] = fmaf(dk, h[1], sa[i].y); h[2] = fmaf(dk, h[2], sa[i].z); h[3] = fmaf(dk, h[3], sa[i].w);
-                h[4] = fmaf(dk, h[4], sb[i].x); h[5] = fmaf(dk, h[5], sb[i].y); h[6] = fmaf(dk, h[6], sb[i].z); h[7] = fmaf(dk, h[7], sb[i].w);
+                h = make_float4(fmaf(dk, h.x, sv[i].x), fmaf(dk, h.y, sv[i].y), fmaf(dk, h.z, sv[i].z), fmaf(dk, h.w, sv[i].w));
             }
         }
     }
     if (fslot < 0) return;
-    if (nck > 0 || fslot != islot) {
-        float4* dst = reinterpret_cast<float4*>(p.pool.ssm + (size_t)fslot * p.pool.ssm_slot_stride + (size_t)d * N + g * 8);
-        dst[0] = make_float4(h[0], h[1], h[2], h[3]);
-        dst[1] = make_float4(h[4], h[5], h[6], h[7]);
-    }
-    if (nck == 0 && fslot != islot && g == 0) {   // a sequence without tokens: its window moves with its state
+    if (nck > 0 || fslot != islot) *reinterpret_cast<float4*>(p.pool.ssm + (size_t)fslot * p.pool.ssm_slot_stride + (size_t)d * N + n0) = h;
+    if (nck == 0 && fslot != islot && g == 0 && sub == 0) {   // a sequence without tokens: its window moves with its state
         __nv_bfloat16* dc = static_cast<__nv_bfloat16*>(p.pool.conv) + (size_t)fslot * p.pool.conv_slot_stride;
         const __nv_bfloat16* sc = islot >= 0 ? static_cast<const __nv_bfloat16*>(p.pool.conv) + (size_t)islot * p.pool.conv_slot_stride : nullptr;
         for (int j = 0; j < kW - 1; ++j) dc[(size_t)j * D + d] = sc ? sc[(size_t)j * D + d] : __float2bfloat16_rn(0.0f);
@@ -403,10 +418,13 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
     ScanSmem& sm = *reinterpret_cast<ScanSmem*>(s_raw + ((128u - (smem_u32(s_raw) & 127u)) & 127u));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads;
+    grid_release_dependents();
+    // Offsets, slots and the C / B rows are inputs of the call (complete before its first kernel let the others start): the
+    // look-ups and the copies of C and B run while the kernels ahead are still at work.
     const ChunkInfo ci = find_chunk(p.cu, p.n_seq, p.T, Q, cidx);
-    if (ci.seq < 0) return;
+    if (ci.seq < 0) { grid_wait(); return; }
     const int islot = load_slot(p.init_slot, ci.seq), fslot = load_slot(p.final_slot, ci.seq);
-    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) return;
+    if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) { grid_wait(); return; }
     const int rows = ci.t1 - ci.t0;
     const size_t ch_head = (size_t)cidx * H + head;
     __nv_bfloat16 (*Ct)[Q][8] = reinterpret_cast<__nv_bfloat16 (*)[Q][8]>(sm.regA);
@@ -427,12 +445,15 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
             tma_box(&Ct[c][0][0], &maps.C, c * 8, ci.t0, &sm.bar_in);
             tma_box(&Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_in);
         }
-        bulk_load(hin, p.ws_hin + ch_head * 2 * N * P, 2 * N * P * 2, &sm.bar_in);
-        bulk_load(sm.csl, p.ws_csl + ch_head * Q, Q * 4, &sm.bar_in);
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 256); tc_fence_before(); }
     __syncthreads();
     tc_fence_after();
+    grid_wait();   // the incoming states and the running decays are the work of the kernels just before
+    if (tid == 0) {
+        bulk_load(hin, p.ws_hin + ch_head * 2 * N * P, 2 * N * P * 2, &sm.bar_in);
+        bulk_load(sm.csl, p.ws_csl + ch_head * Q, Q * 4, &sm.bar_in);
+    }
     const uint32_t tmem = sm.tmem_base;
     const uint32_t tG = tmem, tYi = tmem + 128, tYx = tmem + 192;   // accumulator columns: G, Y inside the chunk, C H_in^T
 
@@ -552,7 +573,27 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
 
 template <typename K>
 cudaError_t allow_smem(K kernel, size_t bytes) {
+    // two blocks of ~100 KB per SM: ask for the largest shared-memory carve-out up front, so that the second block of
+    // an SM does not wait for the split to be changed
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+// Launch with programmatic stream serialisation: the kernel may begin before the one ahead of it has finished.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 }  // namespace
@@ -560,14 +601,14 @@ cudaError_t allow_smem(K kernel, size_t bytes) {
 cudaError_t launch_ssd_prefill(const SsdPrefillArgs& p, const SsdMaps& maps, cudaStream_t st) {
     const int H = p.L.n_heads;
     cudaError_t e;
-    constexpr size_t smem1 = sizeof(StateSmem) + 1024, smem3 = sizeof(ScanSmem) + 128;
+    constexpr size_t smem1 = sizeof(StateSmem) + 128, smem3 = sizeof(ScanSmem) + 128;
     if ((e = allow_smem(ssd_chunk_state_kernel, smem1)) != cudaSuccess) return e;
     if ((e = allow_smem(ssd_chunk_scan_kernel, smem3)) != cudaSuccess) return e;
     dim3 grid(H, p.n_chunks_bound);
-    ssd_chunk_state_kernel<<<grid, kThreads, smem1, st>>>(p, maps);
-    dim3 g2((p.L.d_inner * (N / 8) + 127) / 128, p.n_seq);
-    ssd_state_passing_kernel<<<g2, 128, 0, st>>>(p);
-    ssd_chunk_scan_kernel<<<grid, kThreads, smem3, st>>>(p, maps);
+    if ((e = launch_pdl(ssd_chunk_state_kernel, grid, kThreads, smem1, st, p, maps)) != cudaSuccess) return e;
+    dim3 g2((p.L.d_inner * (N / 4) + kPassThreads - 1) / kPassThreads, p.n_seq);
+    if ((e = launch_pdl(ssd_state_passing_kernel, g2, kPassThreads, 0, st, p)) != cudaSuccess) return e;
+    if ((e = launch_pdl(ssd_chunk_scan_kernel, grid, kThreads, smem3, st, p, maps)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
