@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(kThreads, 3) ssd_chunk_state_kernel(const SsdP
 // Thread = (channel d, 4 states); a lane pair covers one 16-byte unit of the operand.  Walks the sequence's chunks in order:
 // writes the chunk's incoming state as bf16 (a value and a remainder) in the operand layout [state group][channel of the
 // head][8], then h <- exp(chunk decay) h + S.
-constexpr int kPassThreads = 128;
+constexpr int kPassThreads = 256;
 constexpr int kPassBatch = 16;   // chunks whose summaries are in flight together
 
 __global__ void __launch_bounds__(kPassThreads) ssd_state_passing_kernel(const SsdPrefillArgs p) {
@@ -407,7 +407,7 @@ struct ScanSmem {
     unsigned char regB[N / 8 * Q * 16];   // B rows [N/8][Q][8] bf16 (K-major operand)  ->  masked G [Q/8][Q][8] (K-major over the source token)
     unsigned char regH[2 * N * P * 2];    // incoming state [2][N/8][P][8] bf16 (value, remainder; K-major operands)  ->  z box [Q][P] bf16
     float csl[Q];                         // running log2-decay of the chunk's rows (from kernel 1)
-    uint64_t bar_in, bar_late, bar_g, bar_y;
+    uint64_t bar_cb, bar_in, bar_late, bar_g, bar_y;
     uint32_t tmem_base;
 };
 static_assert(sizeof(float) * Q * (P + 1) <= 2 * (N / 8 * Q * 16), "the y staging rows must fit the two operand tiles they lie over");
@@ -437,39 +437,49 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
     float (*ystage)[P + 1] = reinterpret_cast<float (*)[P + 1]>(sm.regA);   // runs on into regB
 
     if (tid == 0) {
-        mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_late, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_y, 1);
+        mbar_init(&sm.bar_cb, 1); mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_late, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_y, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        mbar_expect_tx(&sm.bar_in, 2 * Q * N * 2 + 2 * N * P * 2 + Q * 4);
+        mbar_expect_tx(&sm.bar_cb, 2 * Q * N * 2);
 #pragma unroll
         for (int c = 0; c < N / 8; ++c) {
-            tma_box(&Ct[c][0][0], &maps.C, c * 8, ci.t0, &sm.bar_in);
-            tma_box(&Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_in);
+            tma_box(&Ct[c][0][0], &maps.C, c * 8, ci.t0, &sm.bar_cb);
+            tma_box(&Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_cb);
         }
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 256); tc_fence_before(); }
     __syncthreads();
     tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const uint32_t tG = tmem, tYi = tmem + 128, tYx = tmem + 192;   // accumulator columns: G, Y inside the chunk, C H_in^T
+    // Operand descriptors are built once; an instruction's descriptor is a base plus the step along the contraction index
+    // (the start-address field counts 16-byte units and cannot carry out of its 14 bits: shared memory ends below 256 KB).
+    const uint64_t dC = operand_desc(smem_u32(sm.regA), kColBytes, 128), dB = operand_desc(smem_u32(sm.regB), kColBytes, 128);
+    const uint64_t dH = operand_desc(smem_u32(hin), kHinColBytes, 128), dX = operand_desc(smem_u32(xd), 128, kXdColBytes);
+
+    // G = C B^T needs inputs of the call only: it is issued while the kernels ahead are still at work.
+    const bool cb_ok = mbar_wait_bounded(&sm.bar_cb, 0u);
+    if (cb_ok && tid == 0) {
+        tc_fence_after();
+        constexpr uint32_t idG = instr_desc(Q, false, false);
+#pragma unroll
+        for (int k = 0; k < N / 16; ++k)   // G[t][s] = sum_n C[t][n] B[s][n]
+            mma_bf16(tG, dC + (uint64_t)(k * 2 * kColBytes >> 4), dB + (uint64_t)(k * 2 * kColBytes >> 4), idG, k > 0);
+    }
     grid_wait();   // the incoming states and the running decays are the work of the kernels just before
     if (tid == 0) {
+        mbar_expect_tx(&sm.bar_in, 2 * N * P * 2 + Q * 4);
         bulk_load(hin, p.ws_hin + ch_head * 2 * N * P, 2 * N * P * 2, &sm.bar_in);
         bulk_load(sm.csl, p.ws_csl + ch_head * Q, Q * 4, &sm.bar_in);
     }
-    const uint32_t tmem = sm.tmem_base;
-    const uint32_t tG = tmem, tYi = tmem + 128, tYx = tmem + 192;   // accumulator columns: G, Y inside the chunk, C H_in^T
 
-    const bool ok = mbar_wait_bounded(&sm.bar_in, 0u);
+    const bool ok = cb_ok && mbar_wait_bounded(&sm.bar_in, 0u);
     if (ok && tid == 0) {
         tc_fence_after();
-        const uint32_t c0 = smem_u32(sm.regA), b0 = smem_u32(sm.regB), h0 = smem_u32(hin);
-        constexpr uint32_t idG = instr_desc(Q, false, false), idX = instr_desc(P, false, false);
-#pragma unroll
-        for (int k = 0; k < N / 16; ++k)   // G[t][s] = sum_n C[t][n] B[s][n]
-            mma_bf16(tG, operand_desc(c0 + k * 2 * kColBytes, kColBytes, 128), operand_desc(b0 + k * 2 * kColBytes, kColBytes, 128), idG, k > 0);
+        constexpr uint32_t idX = instr_desc(P, false, false);
 #pragma unroll
         for (int k = 0; k < 2 * (N / 16); ++k) {   // Yx[t][p] = sum_n C[t][n] h_in[p][n], value then remainder
             const int kk = k % (N / 16), part = k / (N / 16);
-            mma_bf16(tYx, operand_desc(c0 + kk * 2 * kColBytes, kColBytes, 128),
-                     operand_desc(h0 + part * (N * P * 2) + kk * 2 * kHinColBytes, kHinColBytes, 128), idX, k > 0);
+            mma_bf16(tYx, dC + (uint64_t)(kk * 2 * kColBytes >> 4), dH + (uint64_t)((part * (N * P * 2) + kk * 2 * kHinColBytes) >> 4), idX, k > 0);
         }
         mma_commit(&sm.bar_g);
     }
@@ -516,11 +526,10 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
     const bool all_ok = !__syncthreads_or(!late_ok);
     if (all_ok && tid == 0) {
         tc_fence_after();
-        const uint32_t m0 = smem_u32(sm.regB), x0 = smem_u32(xd);
         constexpr uint32_t idY = instr_desc(P, false, true);
 #pragma unroll
-        for (int k = 0; k < Q / 16; ++k)   // Yi[t][p] = sum_s M[t][s] Xd[s][p]
-            mma_bf16(tYi, operand_desc(m0 + k * 2 * kColBytes, kColBytes, 128), operand_desc(x0 + k * 256, 128, kXdColBytes), idY, k > 0);
+        for (int k = 0; k < Q / 16; ++k)   // Yi[t][p] = sum_s M[t][s] Xd[s][p]; the masked G lies where the B rows were
+            mma_bf16(tYi, dB + (uint64_t)(k * 2 * kColBytes >> 4), dX + (uint64_t)(k * 256 >> 4), idY, k > 0);
         mma_commit(&sm.bar_y);
     }
     // skip term inputs of the warp's rows travel while the product runs: u of this lane's channel pair (from kernel 1)
@@ -563,7 +572,8 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
         }
     } else if (tid == 0) {
         flag(p.dev_status, MDRAFT_DEV_WAIT_EXPIRED);
-        if (!ok) mbar_wait_bounded(&sm.bar_in, 0u);   // copies target this block's shared memory: one more bounded chance
+        if (!cb_ok) mbar_wait_bounded(&sm.bar_cb, 0u);   // copies target this block's shared memory: one more bounded chance
+        if (!ok) mbar_wait_bounded(&sm.bar_in, 0u);
         if (g_ok && !late_ok) mbar_wait_bounded(&sm.bar_late, 0u);
     }
     tc_fence_before();
