@@ -407,7 +407,7 @@ struct ScanSmem {
     unsigned char regB[N / 8 * Q * 16];   // B rows [N/8][Q][8] bf16 (K-major operand)  ->  masked G [Q/8][Q][8] (K-major over the source token)
     unsigned char regH[2 * N * P * 2];    // incoming state [2][N/8][P][8] bf16 (value, remainder; K-major operands)  ->  z box [Q][P] bf16
     float csl[Q];                         // running log2-decay of the chunk's rows (from kernel 1)
-    uint64_t bar_cb, bar_in, bar_late, bar_g, bar_y;
+    uint64_t bar_cb, bar_in, bar_late, bar_g, bar_x, bar_y;
     uint32_t tmem_base;
 };
 static_assert(sizeof(float) * Q * (P + 1) <= 2 * (N / 8 * Q * 16), "the y staging rows must fit the two operand tiles they lie over");
@@ -437,7 +437,7 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
     float (*ystage)[P + 1] = reinterpret_cast<float (*)[P + 1]>(sm.regA);   // runs on into regB
 
     if (tid == 0) {
-        mbar_init(&sm.bar_cb, 1); mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_late, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_y, 1);
+        mbar_init(&sm.bar_cb, 1); mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_late, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_x, 1); mbar_init(&sm.bar_y, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         mbar_expect_tx(&sm.bar_cb, 2 * Q * N * 2);
 #pragma unroll
@@ -464,6 +464,7 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
 #pragma unroll
         for (int k = 0; k < N / 16; ++k)   // G[t][s] = sum_n C[t][n] B[s][n]
             mma_bf16(tG, dC + (uint64_t)(k * 2 * kColBytes >> 4), dB + (uint64_t)(k * 2 * kColBytes >> 4), idG, k > 0);
+        mma_commit(&sm.bar_g);
     }
     grid_wait();   // the incoming states and the running decays are the work of the kernels just before
     if (tid == 0) {
@@ -481,15 +482,10 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
             const int kk = k % (N / 16), part = k / (N / 16);
             mma_bf16(tYx, dC + (uint64_t)(kk * 2 * kColBytes >> 4), dH + (uint64_t)((part * (N * P * 2) + kk * 2 * kHinColBytes) >> 4), idX, k > 0);
         }
-        mma_commit(&sm.bar_g);
+        mma_commit(&sm.bar_x);
     }
+    // The mask needs G and the decays only: it is written while C H_in^T runs.
     const bool g_ok = ok && mbar_wait_bounded(&sm.bar_g, 0u);
-    if (g_ok && tid == 0) {
-        // both products that read C and the incoming state are complete: their tiles take Xd and the z box
-        mbar_expect_tx(&sm.bar_late, kXdBytes + Q * P * 2);
-        bulk_load(xd, p.ws_xd + ch_head * (kXdBytes / 2), kXdBytes, &sm.bar_late);
-        tma_box(zs, &maps.z, head * P, ci.t0, &sm.bar_late);
-    }
     if (g_ok) {
         tc_fence_after();
         // row t of G, masked: M[t][s] = G[t][s] exp(cs_t - cs_s) for s <= t, else 0; written over the B boxes (G is complete).
@@ -519,6 +515,12 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
             for (int u4 = 0; u4 < 4; ++u4)
                 *reinterpret_cast<uint4*>(&Mt[cb * 4 + u4][row][0]) = make_uint4(packed[4 * u4], packed[4 * u4 + 1], packed[4 * u4 + 2], packed[4 * u4 + 3]);
         }
+    }
+    // Warp 4 has only zeros to write above.  Once C H_in^T is complete, the tiles it read take Xd and the z box.
+    if (warp == 4 && g_ok && mbar_wait_bounded(&sm.bar_x, 0u) && lane == 0) {
+        mbar_expect_tx(&sm.bar_late, kXdBytes + Q * P * 2);
+        bulk_load(xd, p.ws_xd + ch_head * (kXdBytes / 2), kXdBytes, &sm.bar_late);
+        tma_box(zs, &maps.z, head * P, ci.t0, &sm.bar_late);
     }
     const bool late_ok = g_ok && mbar_wait_bounded(&sm.bar_late, 0u);
     fence_async_smem();
