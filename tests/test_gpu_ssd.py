@@ -78,6 +78,16 @@ def test_ssd_prefill_matches_oracle(Dn, lens, init):
     assert np.array_equal(g_conv, o_conv), "conv window must be an exact copy of the last raw inputs"
 
 
+def test_ssd_prefill_at_the_timed_shape():
+    """2048 tokens x 1536 channels (24 heads), one sequence given without offsets, no starting slot: the call bench.py times."""
+    cfg, prm, arrs, cu = make(1536, [2048], seed=2)
+    g_out, g_conv, g_h = run_gpu(prm, arrs, cu, no_offsets=True)
+    o_out, o_conv, o_h = oracle.ssd_prefill(oracle.ssd_layer_from_params(prm), *arrs, cu_seqlens=cu)
+    assert_close(g_out, o_out, TOL["bf16"], "out")
+    assert_close(g_h, o_h, TOL_STATE, "final SSM state")
+    assert np.array_equal(g_conv, o_conv)
+
+
 def test_ssd_prefill_in_pieces_equals_whole():
     """Encode 300 tokens at once, and as 128 + 172 through the slot: the same outputs and state within rounding of
     the different chunk boundaries (chunks 128/128/44 against 128 | 128/44: here identical cuts, so bit for bit)."""
