@@ -8,15 +8,16 @@
 //     S   = sum_s exp(cs_end - cs_s) Delta_s u_s (x) B_s                (what the chunk adds to a zero state)
 //     h_out = exp(cs_end) h_in + S
 //
-// Three stream-ordered kernels, none waiting on another block:
+// Three kernels, none waiting on another block, chained by programmatic dependent launch: the first waits for everything
+// ahead of the call and then lets the others start, so that they may read the call's inputs before their own wait.
 //   1. ssd_chunk_state: per (head, chunk) conv + SiLU, step sizes and running decays, then S^T = B^T Xw on the tensor
 //      cores (tcgen05.mma, bf16 operands, fp32 accumulator in tensor memory); Xw is split into a bf16 value and a bf16
 //      remainder (two products into one accumulator) so that the state keeps fp32-level accuracy.  What kernel 3 needs
 //      of this work is handed over through the workspace: Xd = Delta u already in operand layout, u, and the running
 //      log-decays of the chunk's rows; the sequence's last chunk also leaves the conv window.
-//   2. ssd_state_passing: per (channel, 8 states) the chunk states of a sequence are chained in token order; every
+//   2. ssd_state_passing: per (channel, 4 states) the chunk states of a sequence are chained in token order; every
 //      chunk's incoming state is left in the operand layout the next kernel wants, the final state goes to its slot.
-//   3. ssd_chunk_scan: per (head, chunk) G = C B^T, the causal decay mask applied to G on its way from tensor memory to
+//   3. ssd_chunk_scan: per (head, chunk) G = C B^T (issued before the kernel's wait: inputs only), the causal decay mask applied to G on its way from tensor memory to
 //      shared memory, Y = (G o L) Xd and C H_in^T on the tensor cores, then skip term, gate and store.  It touches no
 //      x, dt or conv weight: its shared memory is three operand tiles, so that two blocks share an SM.
 //
