@@ -473,6 +473,14 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
         bulk_load(hin, p.ws_hin + ch_head * 2 * N * P, 2 * N * P * 2, &sm.bar_in);
         bulk_load(sm.csl, p.ws_csl + ch_head * Q, Q * 4, &sm.bar_in);
     }
+    // skip term inputs of the warp's rows (u of this lane's channel pair, from kernel 1): requested now, used at the very end
+    const int d = head * P + 2 * lane;
+    uint32_t uraw[kRowsPerWarp];
+#pragma unroll
+    for (int i = 0; i < kRowsPerWarp; ++i) {
+        const int r = warp * kRowsPerWarp + i;
+        uraw[i] = r < rows ? *reinterpret_cast<const uint32_t*>(p.ws_u + (size_t)(ci.t0 + r) * p.L.d_inner + d) : 0u;
+    }
 
     const bool ok = cb_ok && mbar_wait_bounded(&sm.bar_in, 0u);
     if (ok && tid == 0) {
@@ -534,14 +542,6 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
         for (int k = 0; k < Q / 16; ++k)   // Yi[t][p] = sum_s M[t][s] Xd[s][p]; the masked G lies where the B rows were
             mma_bf16(tYi, dB + (uint64_t)(k * 2 * kColBytes >> 4), dX + (uint64_t)(k * 256 >> 4), idY, k > 0);
         mma_commit(&sm.bar_y);
-    }
-    // skip term inputs of the warp's rows travel while the product runs: u of this lane's channel pair (from kernel 1)
-    const int d = head * P + 2 * lane;
-    uint32_t uraw[kRowsPerWarp];
-#pragma unroll
-    for (int i = 0; i < kRowsPerWarp; ++i) {
-        const int r = warp * kRowsPerWarp + i;
-        uraw[i] = (all_ok && r < rows) ? *reinterpret_cast<const uint32_t*>(p.ws_u + (size_t)(ci.t0 + r) * p.L.d_inner + d) : 0u;
     }
     bool y_ok = all_ok && mbar_wait_bounded(&sm.bar_y, 0u);
     if (y_ok) {
