@@ -26,7 +26,7 @@ struct SsdLayerDev {
 // TMA descriptors of one context-encode call.
 struct SsdMaps {
     CUtensorMap x, z;   // (T, D) activations, boxes of 64 channels x 128 tokens
-    CUtensorMap B, C;   // (T, N) activations, boxes of 8 states x 128 tokens (one 16-byte column of an operand)
+    CUtensorMap B, C;   // (T, N) activations as (8 states, T, N / 8): one box of 8 x 128 x 16 is a whole operand tile [N / 8][128][8]
 };
 
 struct SsdPrefillArgs {

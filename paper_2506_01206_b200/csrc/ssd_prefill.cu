@@ -64,6 +64,12 @@ __device__ __forceinline__ void tma_box(void* dst, const CUtensorMap* map, int c
                  "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(row), "r"(smem_u32(bar))
                  : "memory");
 }
+// One 128 x 128 tile of B or C (rows `row` ..) as [column group][row][8]: see the descriptor's set-up.
+__device__ __forceinline__ void tma_operand_tile(void* dst, const CUtensorMap* map, int row, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(smem_u32(dst)),
+                 "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(0), "r"(smem_u32(bar))
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
                  "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar)) : "memory");
@@ -215,7 +221,7 @@ __device__ __forceinline__ void conv_rows(const uint32_t (&xr)[kRowsPerWarp + 3]
 
 // ---------------------------------------------------------------- kernel 1: what a chunk adds to a zero state
 struct StateSmem {
-    __nv_bfloat16 Bt[N / 8][Q][8];                        // B rows of the chunk, one TMA box per 8 states
+    __nv_bfloat16 Bt[N / 8][Q][8];                        // B rows of the chunk (one TMA request)
     unsigned char xw_hi[(P / 8) * kXdColBytes];           // Xw = Delta exp(cs_end - cs) u, bf16 value ...
     // ... and bf16 remainder, which takes the place of the x tile (3 rows before the chunk + the x box) once every thread
     // holds its rows of x in registers
@@ -251,8 +257,7 @@ __global__ void __launch_bounds__(kThreads, 3) ssd_chunk_state_kernel(const SsdP
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         mbar_expect_tx(&sm.bar_tma, Q * P * 2 + Q * N * 2);
         tma_box(xs_ext + 3 * P, &maps.x, head * P, ci.t0, &sm.bar_tma);
-#pragma unroll
-        for (int c = 0; c < N / 8; ++c) tma_box(&sm.Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_tma);
+        tma_operand_tile(&sm.Bt[0][0][0], &maps.B, ci.t0, &sm.bar_tma);
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 64); tc_fence_before(); }
     load_halo(xs_ext, p, ci, head, islot);
@@ -441,11 +446,8 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
         mbar_init(&sm.bar_cb, 1); mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_late, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_x, 1); mbar_init(&sm.bar_y, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         mbar_expect_tx(&sm.bar_cb, 2 * Q * N * 2);
-#pragma unroll
-        for (int c = 0; c < N / 8; ++c) {
-            tma_box(&Ct[c][0][0], &maps.C, c * 8, ci.t0, &sm.bar_cb);
-            tma_box(&Bt[c][0][0], &maps.B, c * 8, ci.t0, &sm.bar_cb);
-        }
+        tma_operand_tile(&Ct[0][0][0], &maps.C, ci.t0, &sm.bar_cb);
+        tma_operand_tile(&Bt[0][0][0], &maps.B, ci.t0, &sm.bar_cb);
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 256); tc_fence_before(); }
     __syncthreads();
