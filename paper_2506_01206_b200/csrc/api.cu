@@ -466,6 +466,19 @@ bool encode_ssd_operand(CUtensorMap* m, const void* base, int64_t rows, int64_t 
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Descriptor of a (rows x 128) row-major bf16 matrix read in boxes of 64 columns x 128 rows that land in shared memory as
+// rows of 128 bytes, 16-byte units XOR-ed with the row index (the tensor core's 128-byte-swizzled K-major operand layout).
+bool encode_ssd_swizzled(CUtensorMap* m, const void* base, int64_t rows, int64_t ld) {
+    PFN_cuTensorMapEncodeTiled enc = tensor_map_encoder();
+    if (!enc) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)kSsdN, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kSsdQ};
+    cuuint32_t estride[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 extern "C" {
@@ -523,7 +536,8 @@ int mdraft_ssd_prefill(const mdraft_ssd_layer* layer, const mdraft_cache* cache,
     memset(&maps, 0, sizeof(maps));
     if (have_rows) {
         if (!encode_ssd_matrix(&maps.x, x, total_tokens, D, ldx, kSsdP) || !encode_ssd_matrix(&maps.z, z, total_tokens, D, ldz, kSsdP) ||
-            !encode_ssd_operand(&maps.B, B, total_tokens, ldb) || !encode_ssd_operand(&maps.C, C, total_tokens, ldc))
+            !encode_ssd_operand(&maps.B, B, total_tokens, ldb) || !encode_ssd_swizzled(&maps.Bs, B, total_tokens, ldb) ||
+            !encode_ssd_swizzled(&maps.Cs, C, total_tokens, ldc))
             return MDRAFT_ERR_CUDA;
     }
     return launch_ssd_prefill(a, maps, static_cast<cudaStream_t>(stream)) == cudaSuccess ? MDRAFT_OK : MDRAFT_ERR_CUDA;

@@ -108,6 +108,13 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t saddr, uint32_t lead, 
     return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lead >> 4) & 0x3FFFu) << 16) | ((uint64_t)((stride >> 4) & 0x3FFFu) << 32) |
            (1ull << 46);
 }
+// The same for a K-major operand in the 128-byte-swizzled layout (rows of 64 values = 128 bytes, 8 rows = one 1024-byte
+// group, 16-byte units XOR-ed with the row index; the tile starts on a 1024-byte boundary): the stride field is the step
+// between groups of 8 rows, the leading field is not used, and a step of 16 values along the contraction index is 32 bytes
+// added to the start address.
+__device__ __forceinline__ uint64_t operand_desc_sw128(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n; bit 15 / 16 = A / B operand is MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn, bool b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
@@ -409,8 +416,8 @@ __global__ void __launch_bounds__(kPassThreads) ssd_state_passing_kernel(const S
 //   region H: incoming state, value + remainder        ->  the z box (fetched once C H_in^T is done)
 //   regions A + B                                       ->  y rows on their way from accumulator lanes to channel-contiguous stores
 struct ScanSmem {
-    unsigned char regA[N / 8 * Q * 16];   // C rows [N/8][Q][8] bf16 (K-major operand)  ->  Xd [(P/8)][Q + 1 unit][8] (MN-major operand, from kernel 1)
-    unsigned char regB[N / 8 * Q * 16];   // B rows [N/8][Q][8] bf16 (K-major operand)  ->  masked G [Q/8][Q][8] (K-major over the source token)
+    unsigned char regA[N / 8 * Q * 16];   // C rows [2][Q][64] bf16, 128-byte swizzle (K-major operand)  ->  Xd [(P/8)][Q + 1 unit][8] (MN-major operand, from kernel 1)
+    unsigned char regB[N / 8 * Q * 16];   // B rows [2][Q][64] bf16, 128-byte swizzle (K-major operand)  ->  masked G [Q/8][Q][8] (K-major over the source token)
     unsigned char regH[2 * N * P * 2];    // incoming state [2][N/8][P][8] bf16 (value, remainder; K-major operands)  ->  z box [Q][P] bf16
     float csl[Q];                         // running log2-decay of the chunk's rows (from kernel 1)
     uint64_t bar_cb, bar_in, bar_late, bar_g, bar_x, bar_y;
@@ -421,7 +428,7 @@ static_assert((P / 8) * kXdColBytes <= N / 8 * Q * 16 && Q * P * 2 <= 2 * N * P 
 
 __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
     extern __shared__ __align__(1024) unsigned char s_raw[];
-    ScanSmem& sm = *reinterpret_cast<ScanSmem*>(s_raw + ((128u - (smem_u32(s_raw) & 127u)) & 127u));
+    ScanSmem& sm = *reinterpret_cast<ScanSmem*>(s_raw + ((1024u - (smem_u32(s_raw) & 1023u)) & 1023u));   // swizzled tiles start on 1024-byte boundaries
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads;
     grid_release_dependents();
@@ -433,8 +440,6 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
     if (islot >= p.pool.n_slots || fslot >= p.pool.n_slots) { grid_wait(); return; }
     const int rows = ci.t1 - ci.t0;
     const size_t ch_head = (size_t)cidx * H + head;
-    __nv_bfloat16 (*Ct)[Q][8] = reinterpret_cast<__nv_bfloat16 (*)[Q][8]>(sm.regA);
-    __nv_bfloat16 (*Bt)[Q][8] = reinterpret_cast<__nv_bfloat16 (*)[Q][8]>(sm.regB);
     __nv_bfloat16 (*Mt)[Q][8] = reinterpret_cast<__nv_bfloat16 (*)[Q][8]>(sm.regB);
     unsigned char* xd = sm.regA;
     constexpr uint32_t kXdBytes = (P / 8) * kXdColBytes;
@@ -446,8 +451,11 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
         mbar_init(&sm.bar_cb, 1); mbar_init(&sm.bar_in, 1); mbar_init(&sm.bar_late, 1); mbar_init(&sm.bar_g, 1); mbar_init(&sm.bar_x, 1); mbar_init(&sm.bar_y, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         mbar_expect_tx(&sm.bar_cb, 2 * Q * N * 2);
-        tma_operand_tile(&Ct[0][0][0], &maps.C, ci.t0, &sm.bar_cb);
-        tma_operand_tile(&Bt[0][0][0], &maps.B, ci.t0, &sm.bar_cb);
+        // two boxes of 64 states x 128 tokens per matrix
+        tma_box(sm.regA, &maps.Cs, 0, ci.t0, &sm.bar_cb);
+        tma_box(sm.regA + Q * 128, &maps.Cs, 64, ci.t0, &sm.bar_cb);
+        tma_box(sm.regB, &maps.Bs, 0, ci.t0, &sm.bar_cb);
+        tma_box(sm.regB + Q * 128, &maps.Bs, 64, ci.t0, &sm.bar_cb);
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 256); tc_fence_before(); }
     __syncthreads();
@@ -456,8 +464,12 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
     const uint32_t tG = tmem, tYi = tmem + 128, tYx = tmem + 192;   // accumulator columns: G, Y inside the chunk, C H_in^T
     // Operand descriptors are built once; an instruction's descriptor is a base plus the step along the contraction index
     // (the start-address field counts 16-byte units and cannot carry out of its 14 bits: shared memory ends below 256 KB).
-    const uint64_t dC = operand_desc(smem_u32(sm.regA), kColBytes, 128), dB = operand_desc(smem_u32(sm.regB), kColBytes, 128);
+    // C and B rows: swizzled tiles; contraction step k (16 states) starts 32 bytes further on inside a half of 64 states,
+    // the second half lies one 16 KB box further on.  The masked G that replaces the B rows is un-swizzled.
+    const uint64_t dC = operand_desc_sw128(smem_u32(sm.regA)), dB = operand_desc_sw128(smem_u32(sm.regB));
+    const uint64_t dM = operand_desc(smem_u32(sm.regB), kColBytes, 128);
     const uint64_t dH = operand_desc(smem_u32(hin), kHinColBytes, 128), dX = operand_desc(smem_u32(xd), 128, kXdColBytes);
+    auto kstep = [](int k) { return (uint64_t)(((k >> 2) * (Q * 128) + (k & 3) * 32) >> 4); };
 
     // G = C B^T needs inputs of the call only: it is issued while the kernels ahead are still at work.
     const bool cb_ok = mbar_wait_bounded(&sm.bar_cb, 0u);
@@ -466,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
         constexpr uint32_t idG = instr_desc(Q, false, false);
 #pragma unroll
         for (int k = 0; k < N / 16; ++k)   // G[t][s] = sum_n C[t][n] B[s][n]
-            mma_bf16(tG, dC + (uint64_t)(k * 2 * kColBytes >> 4), dB + (uint64_t)(k * 2 * kColBytes >> 4), idG, k > 0);
+            mma_bf16(tG, dC + kstep(k), dB + kstep(k), idG, k > 0);
         mma_commit(&sm.bar_g);
     }
     grid_wait();   // the incoming states and the running decays are the work of the kernels just before
@@ -491,7 +503,7 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
 #pragma unroll
         for (int k = 0; k < 2 * (N / 16); ++k) {   // Yx[t][p] = sum_n C[t][n] h_in[p][n], value then remainder
             const int kk = k % (N / 16), part = k / (N / 16);
-            mma_bf16(tYx, dC + (uint64_t)(kk * 2 * kColBytes >> 4), dH + (uint64_t)((part * (N * P * 2) + kk * 2 * kHinColBytes) >> 4), idX, k > 0);
+            mma_bf16(tYx, dC + kstep(kk), dH + (uint64_t)((part * (N * P * 2) + kk * 2 * kHinColBytes) >> 4), idX, k > 0);
         }
         mma_commit(&sm.bar_x);
     }
@@ -542,7 +554,7 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
         constexpr uint32_t idY = instr_desc(P, false, true);
 #pragma unroll
         for (int k = 0; k < Q / 16; ++k)   // Yi[t][p] = sum_s M[t][s] Xd[s][p]; the masked G lies where the B rows were
-            mma_bf16(tYi, dB + (uint64_t)(k * 2 * kColBytes >> 4), dX + (uint64_t)(k * 256 >> 4), idY, k > 0);
+            mma_bf16(tYi, dM + (uint64_t)(k * 2 * kColBytes >> 4), dX + (uint64_t)(k * 256 >> 4), idY, k > 0);
         mma_commit(&sm.bar_y);
     }
     bool y_ok = all_ok && mbar_wait_bounded(&sm.bar_y, 0u);
@@ -616,7 +628,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t 
 cudaError_t launch_ssd_prefill(const SsdPrefillArgs& p, const SsdMaps& maps, cudaStream_t st) {
     const int H = p.L.n_heads;
     cudaError_t e;
-    constexpr size_t smem1 = sizeof(StateSmem) + 128, smem3 = sizeof(ScanSmem) + 128;
+    constexpr size_t smem1 = sizeof(StateSmem) + 128, smem3 = sizeof(ScanSmem) + 1024;
     if ((e = allow_smem(ssd_chunk_state_kernel, smem1)) != cudaSuccess) return e;
     if ((e = allow_smem(ssd_chunk_scan_kernel, smem3)) != cudaSuccess) return e;
     dim3 grid(H, p.n_chunks_bound);
