@@ -452,20 +452,6 @@ bool encode_ssd_matrix(CUtensorMap* m, const void* base, int64_t rows, int64_t c
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Descriptor of a (rows x 128) row-major bf16 matrix (B or C) seen as (8 values, rows, 16 groups of 8 columns): one box of
-// 8 x 128 x 16 brings a whole 128 x 128 tile into shared memory as [column group][row][8], which is the tensor core's
-// un-swizzled operand layout, with a single request.
-bool encode_ssd_operand(CUtensorMap* m, const void* base, int64_t rows, int64_t ld) {
-    PFN_cuTensorMapEncodeTiled enc = tensor_map_encoder();
-    if (!enc) return false;
-    cuuint64_t gdim[3] = {8, (cuuint64_t)rows, (cuuint64_t)(kSsdN / 8)};
-    cuuint64_t gstride[2] = {(cuuint64_t)ld * 2, 16};
-    cuuint32_t box[3] = {8, (cuuint32_t)kSsdQ, (cuuint32_t)(kSsdN / 8)};
-    cuuint32_t estride[3] = {1, 1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // Descriptor of a (rows x 128) row-major bf16 matrix read in boxes of 64 columns x 128 rows that land in shared memory as
 // rows of 128 bytes, 16-byte units XOR-ed with the row index (the tensor core's 128-byte-swizzled K-major operand layout).
 bool encode_ssd_swizzled(CUtensorMap* m, const void* base, int64_t rows, int64_t ld) {
@@ -536,7 +522,7 @@ int mdraft_ssd_prefill(const mdraft_ssd_layer* layer, const mdraft_cache* cache,
     memset(&maps, 0, sizeof(maps));
     if (have_rows) {
         if (!encode_ssd_matrix(&maps.x, x, total_tokens, D, ldx, kSsdP) || !encode_ssd_matrix(&maps.z, z, total_tokens, D, ldz, kSsdP) ||
-            !encode_ssd_operand(&maps.B, B, total_tokens, ldb) || !encode_ssd_swizzled(&maps.Bs, B, total_tokens, ldb) ||
+            !encode_ssd_swizzled(&maps.Bs, B, total_tokens, ldb) ||
             !encode_ssd_swizzled(&maps.Cs, C, total_tokens, ldc))
             return MDRAFT_ERR_CUDA;
     }

@@ -26,7 +26,6 @@ struct SsdLayerDev {
 // TMA descriptors of one context-encode call.
 struct SsdMaps {
     CUtensorMap x, z;   // (T, D) activations, boxes of 64 channels x 128 tokens
-    CUtensorMap B;      // (T, N) activations as (8 states, T, N / 8): one box of 8 x 128 x 16 is a whole operand tile [N / 8][128][8]
     CUtensorMap Bs, Cs; // (T, N) activations in boxes of 64 states x 128 tokens, 128-byte swizzle (rows of 128 bytes: full sectors)
 };
 

@@ -23,9 +23,11 @@
 //
 // Operands live in shared memory in the tensor core's canonical un-swizzled layout: 16-byte units of 8 bf16 values,
 // 8 units = one 8 x 8 "core matrix" of 128 contiguous bytes; one descriptor field gives the byte step between core
-// matrices along the contraction index, the other along the row index.  A TMA box of 8 columns x 128 rows of a
-// row-major matrix lands exactly as one column of core matrices, so B and C arrive in operand form without a pass
-// over them, both as "K-major" (G: contraction over the state index) and as "MN-major" (S: contraction over tokens).
+// matrices along the contraction index, the other along the row index.  That is the layout of the operands that threads
+// write (Xw, Xd, the masked G) and of the incoming state.  The B and C rows come by TMA in boxes of 64 states x 128 tokens
+// with the 128-byte swizzle (rows of 128 bytes, 16-byte units XOR-ed with the row index: full sectors on the way in and the
+// tensor core's swizzled operand layout in shared memory), so they arrive in operand form without a pass over them, both as
+// "K-major" (G: contraction over the state index) and as "MN-major" (S: contraction over tokens) - same bytes, two descriptors.
 // All waits on mbarriers are bounded (MDRAFT_DEV_WAIT_EXPIRED); tensor memory is freed on every path.
 #include "chunk_map.cuh"
 #include "common.cuh"
@@ -62,12 +64,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
 __device__ __forceinline__ void tma_box(void* dst, const CUtensorMap* map, int col, int row, uint64_t* bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_u32(dst)),
                  "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(row), "r"(smem_u32(bar))
-                 : "memory");
-}
-// One 128 x 128 tile of B or C (rows `row` ..) as [column group][row][8]: see the descriptor's set-up.
-__device__ __forceinline__ void tma_operand_tile(void* dst, const CUtensorMap* map, int row, uint64_t* bar) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(smem_u32(dst)),
-                 "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(0), "r"(smem_u32(bar))
                  : "memory");
 }
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -114,6 +110,12 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t saddr, uint32_t lead, 
 // added to the start address.
 __device__ __forceinline__ uint64_t operand_desc_sw128(uint32_t saddr) {
     return (uint64_t)((saddr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// The same layout read as an MN-major operand (rows of 64 MN-values, one row per contraction index): `lead` is the step
+// between blocks of 64 MN-values, `stride` the step between groups of 8 contraction indices.
+__device__ __forceinline__ uint64_t operand_desc_sw128_mn(uint32_t saddr, uint32_t lead, uint32_t stride) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lead >> 4) & 0x3FFFu) << 16) | ((uint64_t)((stride >> 4) & 0x3FFFu) << 32) | (1ull << 46) |
+           (2ull << 61);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n; bit 15 / 16 = A / B operand is MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn, bool b_mn) {
@@ -228,7 +230,7 @@ __device__ __forceinline__ void conv_rows(const uint32_t (&xr)[kRowsPerWarp + 3]
 
 // ---------------------------------------------------------------- kernel 1: what a chunk adds to a zero state
 struct StateSmem {
-    __nv_bfloat16 Bt[N / 8][Q][8];                        // B rows of the chunk (one TMA request)
+    unsigned char Bt[Q * N * 2];                          // B rows of the chunk [2][Q][64] bf16, 128-byte swizzle (MN-major operand)
     unsigned char xw_hi[(P / 8) * kXdColBytes];           // Xw = Delta exp(cs_end - cs) u, bf16 value ...
     // ... and bf16 remainder, which takes the place of the x tile (3 rows before the chunk + the x box) once every thread
     // holds its rows of x in registers
@@ -238,11 +240,11 @@ struct StateSmem {
     uint32_t tmem_base;
 };
 static_assert((Q + 3) * P * 2 >= (P / 8) * kXdColBytes, "the remainder operand must fit the x tile it replaces");
-static_assert(3 * (sizeof(StateSmem) + 128 + 1024) <= 227 * 1024, "three blocks per SM");
+static_assert(3 * (sizeof(StateSmem) + 1024 + 1024) <= 227 * 1024, "three blocks per SM");
 
 __global__ void __launch_bounds__(kThreads, 3) ssd_chunk_state_kernel(const SsdPrefillArgs p, const __grid_constant__ SsdMaps maps) {
     extern __shared__ __align__(1024) unsigned char s_raw[];
-    StateSmem& sm = *reinterpret_cast<StateSmem*>(s_raw + ((128u - (smem_u32(s_raw) & 127u)) & 127u));
+    StateSmem& sm = *reinterpret_cast<StateSmem*>(s_raw + ((1024u - (smem_u32(s_raw) & 1023u)) & 1023u));   // the swizzled tile starts on a 1024-byte boundary
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = blockIdx.x, cidx = blockIdx.y, H = p.L.n_heads;
     // The inputs may be the work of the kernel ahead of this call, and the workspace is still being read by the call
@@ -264,7 +266,8 @@ __global__ void __launch_bounds__(kThreads, 3) ssd_chunk_state_kernel(const SsdP
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         mbar_expect_tx(&sm.bar_tma, Q * P * 2 + Q * N * 2);
         tma_box(xs_ext + 3 * P, &maps.x, head * P, ci.t0, &sm.bar_tma);
-        tma_operand_tile(&sm.Bt[0][0][0], &maps.B, ci.t0, &sm.bar_tma);
+        tma_box(sm.Bt, &maps.Bs, 0, ci.t0, &sm.bar_tma);
+        tma_box(sm.Bt + Q * 128, &maps.Bs, 64, ci.t0, &sm.bar_tma);
     }
     if (warp == 0) { tmem_alloc(&sm.tmem_base, 64); tc_fence_before(); }
     load_halo(xs_ext, p, ci, head, islot);
@@ -307,13 +310,15 @@ __global__ void __launch_bounds__(kThreads, 3) ssd_chunk_state_kernel(const SsdP
         tc_fence_after();
         // S^T (n x p) = sum over tokens: A operand = B^T read MN-major out of the TMA boxes, B operand = Xw MN-major.
         constexpr uint32_t idesc = instr_desc(P, true, true);
-        const uint32_t a0 = smem_u32(&sm.Bt[0][0][0]), bh = smem_u32(sm.xw_hi), bl = smem_u32(xw_lo);
+        const uint32_t bh = smem_u32(sm.xw_hi), bl = smem_u32(xw_lo);
+        // B^T: two blocks of 64 states (16 KB apart), 16 tokens per instruction = two groups of 8 rows of 128 bytes
+        const uint64_t dA = operand_desc_sw128_mn(smem_u32(sm.Bt), Q * 128, 1024);
 #pragma unroll
         for (int k = 0; k < Q / 16; ++k)
-            mma_bf16(tmem, operand_desc(a0 + k * 256, 128, kColBytes), operand_desc(bh + k * 256, 128, kXdColBytes), idesc, k > 0);
+            mma_bf16(tmem, dA + (uint64_t)(k * 2048 >> 4), operand_desc(bh + k * 256, 128, kXdColBytes), idesc, k > 0);
 #pragma unroll
         for (int k = 0; k < Q / 16; ++k)
-            mma_bf16(tmem, operand_desc(a0 + k * 256, 128, kColBytes), operand_desc(bl + k * 256, 128, kXdColBytes), idesc, true);
+            mma_bf16(tmem, dA + (uint64_t)(k * 2048 >> 4), operand_desc(bl + k * 256, 128, kXdColBytes), idesc, true);
         mma_commit(&sm.bar_mma);
     }
     bool done = all_ok && mbar_wait_bounded(&sm.bar_mma, 0u);
@@ -628,7 +633,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t 
 cudaError_t launch_ssd_prefill(const SsdPrefillArgs& p, const SsdMaps& maps, cudaStream_t st) {
     const int H = p.L.n_heads;
     cudaError_t e;
-    constexpr size_t smem1 = sizeof(StateSmem) + 128, smem3 = sizeof(ScanSmem) + 1024;
+    constexpr size_t smem1 = sizeof(StateSmem) + 1024, smem3 = sizeof(ScanSmem) + 1024;
     if ((e = allow_smem(ssd_chunk_state_kernel, smem1)) != cudaSuccess) return e;
     if ((e = allow_smem(ssd_chunk_scan_kernel, smem3)) != cudaSuccess) return e;
     dim3 grid(H, p.n_chunks_bound);
