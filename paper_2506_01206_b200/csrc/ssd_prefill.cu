@@ -141,6 +141,14 @@ __device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;
 __device__ __forceinline__ void grid_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// SiLU of the gate input with one special-function instruction instead of two: z sigmoid(z) = 0.5 z (1 + tanh(z / 2)); the
+// approximate tanh is good to about 2^-11, an order below the bf16 rounding of `out`.
+__device__ __forceinline__ float silu_gate(float v) {
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * v));
+    const float h = 0.5f * v;
+    return fmaf(h, t, h);
+}
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 __device__ __forceinline__ uint32_t pack_bf(float lo, float hi) {
@@ -587,8 +595,8 @@ __global__ void __launch_bounds__(kThreads, 2) ssd_chunk_scan_kernel(const SsdPr
             const int r = warp * kRowsPerWarp + i;
             if (r < rows) {
                 const uint32_t zv = zc[r * (P / 2)];
-                const float oa = fmaf(da, bf_lo(uraw[i]), ystage[r][2 * lane]) * silu(bf_lo(zv));
-                const float ob = fmaf(db, bf_hi(uraw[i]), ystage[r][2 * lane + 1]) * silu(bf_hi(zv));
+                const float oa = fmaf(da, bf_lo(uraw[i]), ystage[r][2 * lane]) * silu_gate(bf_lo(zv));
+                const float ob = fmaf(db, bf_hi(uraw[i]), ystage[r][2 * lane + 1]) * silu_gate(bf_hi(zv));
                 *reinterpret_cast<uint32_t*>(p.out + (size_t)(ci.t0 + r) * p.ldo + d) = pack_bf(oa, ob);
             }
         }
