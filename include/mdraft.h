@@ -290,7 +290,8 @@ int mdraft_tree_step_proj(const mdraft_layer *layer, const mdraft_cache *cache, 
  * accumulation): u * Delta and the masked C.B products are rounded to bf16 on the way into a product, so `out`
  * carries a relative error of a few 2^-9 before its own rounding to bf16; the incoming state of a chunk and the
  * operand of the state product are split into a bf16 value plus a bf16 remainder (two products into one
- * accumulator), so what depends on the state, and the state written to the slot, keep fp32-level accuracy.
+ * accumulator), so what depends on the state, and the state written to the slot, keep fp32-level accuracy.  The
+ * encode's gate uses SiLU(z) = z/2 * (1 + tanh(z/2)) with the hardware's approximate tanh (about 2^-11).
  */
 typedef struct {
     int32_t d_inner;        /* D */
